@@ -1,0 +1,154 @@
+/* sasq.h -- C ABI of the B200 (sm_100a) SASQ hot-path library.
+ *
+ * SASQ (Static Activation Scaling for Quantization-aware training) inserts a
+ * fake-quantization operator in front of every frozen linear layer, trains only
+ * the activation quantization factors (Sec. 4.2), and at inference applies the
+ * learned factors statically in front of an integer GEMM (Fig. 1, Eq. 2).
+ *
+ * Notation (Eq. 1):  b = bits, Qn = 2^(b-1), Qp = 2^(b-1) - 1, s = factor.
+ *   inv = fl32(1 / s)            one IEEE fp32 division per factor
+ *   t   = fl32(x * inv)          one fp32 multiply, never fused with anything
+ *   r   = rint(t)                round to nearest, ties to even
+ *   c   = min(max(r, -Qn), Qp)   the integer code of Eq. 1
+ *   m   = (-Qn <= r <= Qp)       Eq. 4: clamp passes the gradient, ends included
+ *
+ * General rules
+ *   - Every data pointer is a DEVICE pointer unless its comment says "host".
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  All work is enqueued on it; no call synchronises except
+ *     sasq_device_status.
+ *   - The caller owns every buffer.  The library allocates no device memory.
+ *   - Tensors are dense, row-major, 16-bit floating point (sasq_dtype_t) and
+ *     16-byte aligned.  Factors are fp32 and live in device memory so that an
+ *     optimizer can update them without a host round trip.
+ *   - A factor may be any finite non-zero fp32 whose reciprocal is finite,
+ *     negative values included (the paper puts no constraint on the update
+ *     range, Sec. 4.2).  A zero / NaN / Inf factor is detected on the device:
+ *     the sticky status word becomes SASQ_ERR_BAD_SCALE and outputs are
+ *     unspecified.
+ *   - Non-finite activations are outside the contract.  What happens anyway:
+ *     +-Inf saturates (m = 0); NaN gives code -Qn, m = 0.
+ *   - Host-detectable errors (NULL or misaligned pointers, sizes, bits,
+ *     workspace too small, wrong device architecture) return a code and launch
+ *     nothing.  There is no CPU fallback.
+ *   - numel == 0 / T == 0 is SASQ_OK without a launch (grad_scale is zeroed
+ *     unless accumulating).
+ */
+#ifndef SASQ_H_
+#define SASQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define SASQ_API __attribute__((visibility("default")))
+#else
+#define SASQ_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SASQ_OK = 0,
+    SASQ_ERR_INVALID_ARG = 1,   /* NULL / misaligned pointer, negative size, bits outside [2, 8] ... */
+    SASQ_ERR_UNSUPPORTED = 2,   /* shape constraint of a kernel not met, or device is not sm_100 */
+    SASQ_ERR_WORKSPACE = 3,     /* workspace NULL or smaller than the matching *_workspace() query */
+    SASQ_ERR_BAD_SCALE = 4,     /* device-detected: factor is 0, NaN, Inf or has a non-finite reciprocal */
+    SASQ_ERR_TIMEOUT = 5,       /* device-detected: a bounded wait inside a kernel gave up */
+    SASQ_ERR_CUDA = 6           /* a CUDA runtime / driver call failed */
+} sasq_status_t;
+
+typedef enum { SASQ_F16 = 0, SASQ_BF16 = 1 } sasq_dtype_t;
+
+/* One tensor of a multi-tensor fake-quant launch (host struct).  y == NULL skips
+ * the forward output; grad_y == grad_x == NULL skips the backward; at least one
+ * part must be present and every descriptor of one call must have the same
+ * parts.  scale_index selects the factor (and the gradient slot) in the arrays
+ * passed to the call; several tensors may share one index, which is how one
+ * factor per decoder layer is expressed. */
+typedef struct {
+    const void* x;        /* [numel] activations */
+    const void* grad_y;   /* [numel] upstream gradient, or NULL */
+    void* y;              /* [numel] fake-quantized output, or NULL */
+    void* grad_x;         /* [numel] input gradient, or NULL (must be non-NULL iff grad_y is) */
+    int64_t numel;
+    int32_t scale_index;
+    int32_t reserved;     /* must be 0 */
+} sasq_qdesc_t;
+
+SASQ_API const char* sasq_status_string(int status);
+
+/* Fake-quant forward (Sec. 4.2: quant, round, clamp, dequant; Eq. 1):
+ *   y[i] = narrow( fl32(c_i * s) ),  one round-to-nearest-even narrowing to `dt`.
+ * x, y: [numel] of `dt`; y may alias x.  scale_dev: one fp32.  bits in [2, 8]. */
+SASQ_API int sasq_fakequant_fwd(const void* x, void* y, int64_t numel, int dt, const float* scale_dev, int bits,
+                       void* stream);
+
+/* Bytes of scratch the backward / fused calls need for a single tensor. */
+SASQ_API size_t sasq_fakequant_bwd_workspace(int64_t numel);
+
+/* Straight-through backward (Eq. 4) and the factor gradient that follows from it
+ * by the chain rule, summed over EVERY element of the tensor:
+ *   grad_x[i]  = m_i ? grad_y[i] : +0                        (bit copy or zero)
+ *   grad_scale = sum_i grad_y[i] * (m_i ? (r_i - t_i) : c_i)  (no normalisation)
+ * The sum is taken as fp32 products, fixed-shape fp32 trees of 8, then double
+ * accumulation per thread, a fixed-order block reduction and a fixed-order
+ * second-stage combine: the result is bit-identical from run to run and within
+ * 1e-4 relative of a double-precision sum.
+ * grad_scale_dev: one fp32, overwritten (accumulate == 0) or added to (!= 0).
+ * workspace: >= sasq_fakequant_bwd_workspace(numel) bytes, 16-byte aligned; its
+ * contents need no initialisation and are garbage afterwards.  Calls that share
+ * a workspace must be ordered on the stream. grad_x may alias grad_y. */
+SASQ_API int sasq_fakequant_bwd(const void* x, const void* grad_y, void* grad_x, float* grad_scale_dev, int accumulate,
+                       int64_t numel, int dt, const float* scale_dev, int bits, void* workspace,
+                       size_t ws_bytes, void* stream);
+
+/* Forward and backward in one pass over x and grad_y (what one scale-only
+ * training step does per quantizer): same results as the two calls above. */
+SASQ_API int sasq_fakequant_fwd_bwd(const void* x, const void* grad_y, void* y, void* grad_x, float* grad_scale_dev,
+                           int accumulate, int64_t numel, int dt, const float* scale_dev, int bits,
+                           void* workspace, size_t ws_bytes, void* stream);
+
+/* Bytes of scratch for a multi-tensor call with n_tensors descriptors. */
+SASQ_API size_t sasq_fakequant_multi_workspace(int n_tensors);
+
+/* Several quantizers in one call (e.g. the seven linear inputs of a decoder
+ * layer).  descs_host: HOST array of n_tensors descriptors, copied into the
+ * launch parameters (it may be freed on return).  scales_dev[n_scales] fp32,
+ * grad_scales_dev[n_scales] fp32 (may be NULL when no descriptor has a backward
+ * part).  Every slot of grad_scales_dev that some descriptor with a backward
+ * part refers to is overwritten (or accumulated into); other slots are left
+ * alone.  A slot shared by several tensors receives the sum over all of them,
+ * combined in descriptor order (one factor per layer). */
+SASQ_API int sasq_fakequant_fwd_bwd_multi(const sasq_qdesc_t* descs_host, int n_tensors, const float* scales_dev,
+                                 float* grad_scales_dev, int n_scales, int accumulate, int dt, int bits,
+                                 void* workspace, size_t ws_bytes, void* stream);
+
+/* Bytes of scratch sasq_static_w8a8_linear needs for this shape (may be 0). */
+SASQ_API size_t sasq_static_w8a8_linear_workspace(int64_t T, int64_t N, int64_t K);
+
+/* Static W8A8 linear (Eq. 1 with the fixed learned factor, then Eq. 2):
+ *   X_int[t,k] = int8(c(x[t,k]))                 no max / scale pass at run time
+ *   acc[t,n]   = sum_k X_int[t,k] * w[n,k]       int32, exact
+ *   y[t,n]     = narrow( fl32(acc) * fl32(s_x * w_scale[n]) (+ bias[n]) )
+ * x: [T, K] of `dt`.  w: [N, K] int8, one row per output channel (the paper's W
+ * is its transpose).  w_scale: [N] fp32 per-output-channel weight factors.
+ * x_scale_dev: one fp32.  bias: [N] of `dt` or NULL (bias is never quantized,
+ * Sec. 3).  y: [T, N] of `dt`.  acc_out: [T, N] int32 or NULL; when given, the
+ * raw accumulators are also written (parity / debugging).
+ * Constraints: K % 16 == 0, N % 8 == 0, K <= 131072 (int32 cannot overflow),
+ * bits in [2, 8]; otherwise SASQ_ERR_UNSUPPORTED. */
+SASQ_API int sasq_static_w8a8_linear(const void* x, const int8_t* w, const float* w_scale, const float* x_scale_dev,
+                            const void* bias, void* y, int32_t* acc_out, int64_t T, int64_t N, int64_t K,
+                            int dt, int bits, void* workspace, size_t ws_bytes, void* stream);
+
+/* Synchronises `stream`, returns the sticky device status word of the current
+ * device (SASQ_OK, SASQ_ERR_BAD_SCALE or SASQ_ERR_TIMEOUT) and clears it. */
+SASQ_API int sasq_device_status(void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SASQ_H_ */

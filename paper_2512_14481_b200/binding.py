@@ -1,0 +1,228 @@
+"""ctypes binding of libsasq_b200.so.  Same names as include/sasq.h.
+
+Every function takes torch CUDA tensors (used purely as device memory), checks
+dtype / device / contiguity, and passes raw pointers and sizes to the library on
+the current torch stream.  A non-zero status raises SasqError.  If the shared
+library is missing or cannot be loaded, import of this module's functions fails
+loudly: there is no CPU or PyTorch fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+__all__ = [
+    "SasqError", "SASQ_F16", "SASQ_BF16", "library_path", "load_library", "sasq_status_string",
+    "sasq_fakequant_fwd", "sasq_fakequant_bwd_workspace", "sasq_fakequant_bwd", "sasq_fakequant_fwd_bwd",
+    "sasq_fakequant_multi_workspace", "sasq_fakequant_fwd_bwd_multi", "sasq_static_w8a8_linear_workspace",
+    "sasq_static_w8a8_linear", "sasq_device_status", "QDesc",
+]
+
+SASQ_F16 = 0
+SASQ_BF16 = 1
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libsasq_b200.so")
+_lib = None
+
+
+class SasqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = int(status)
+        super().__init__(f"{where}: {sasq_status_string(status)} (status {status})")
+
+
+class QDesc(ctypes.Structure):
+    """Mirror of sasq_qdesc_t."""
+    _fields_ = [("x", ctypes.c_void_p), ("grad_y", ctypes.c_void_p), ("y", ctypes.c_void_p),
+                ("grad_x", ctypes.c_void_p), ("numel", ctypes.c_int64), ("scale_index", ctypes.c_int32),
+                ("reserved", ctypes.c_int32)]
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads the CUDA library; raises if it has not been built (python -m paper_2512_14481_b200.build)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError(f"{_LIB_PATH} is missing: build it with `python -m paper_2512_14481_b200.build` "
+                           "(there is no fallback path)")
+    L = ctypes.CDLL(_LIB_PATH)
+    vp, i64, i32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t
+    L.sasq_status_string.restype = ctypes.c_char_p
+    L.sasq_status_string.argtypes = [i32]
+    L.sasq_fakequant_fwd.restype = i32
+    L.sasq_fakequant_fwd.argtypes = [vp, vp, i64, i32, vp, i32, vp]
+    L.sasq_fakequant_bwd_workspace.restype = sz
+    L.sasq_fakequant_bwd_workspace.argtypes = [i64]
+    L.sasq_fakequant_bwd.restype = i32
+    L.sasq_fakequant_bwd.argtypes = [vp, vp, vp, vp, i32, i64, i32, vp, i32, vp, sz, vp]
+    L.sasq_fakequant_fwd_bwd.restype = i32
+    L.sasq_fakequant_fwd_bwd.argtypes = [vp, vp, vp, vp, vp, i32, i64, i32, vp, i32, vp, sz, vp]
+    L.sasq_fakequant_multi_workspace.restype = sz
+    L.sasq_fakequant_multi_workspace.argtypes = [i32]
+    L.sasq_fakequant_fwd_bwd_multi.restype = i32
+    L.sasq_fakequant_fwd_bwd_multi.argtypes = [ctypes.POINTER(QDesc), i32, vp, vp, i32, i32, i32, i32, vp, sz, vp]
+    L.sasq_static_w8a8_linear_workspace.restype = sz
+    L.sasq_static_w8a8_linear_workspace.argtypes = [i64, i64, i64]
+    L.sasq_static_w8a8_linear.restype = i32
+    L.sasq_static_w8a8_linear.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, sz, vp]
+    L.sasq_device_status.restype = i32
+    L.sasq_device_status.argtypes = [vp]
+    _lib = L
+    return L
+
+
+def sasq_status_string(status: int) -> str:
+    return load_library().sasq_status_string(int(status)).decode()
+
+
+# ---------------------------------------------------------------------------
+# marshalling helpers
+# ---------------------------------------------------------------------------
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float16:
+        return SASQ_F16
+    if t.dtype == torch.bfloat16:
+        return SASQ_BF16
+    raise TypeError(f"expected float16 or bfloat16, got {t.dtype}")
+
+
+def _dev(t, name: str, dtype=None):
+    if t is None:
+        return None
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+    return t
+
+
+def _ptr(t) -> int | None:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise SasqError(status, where)
+
+
+def _nbytes(t) -> int:
+    return 0 if t is None else t.numel() * t.element_size()
+
+
+# ---------------------------------------------------------------------------
+# the entry points
+# ---------------------------------------------------------------------------
+def sasq_fakequant_fwd(x: torch.Tensor, y: torch.Tensor, scale: torch.Tensor, bits: int = 8, stream=None) -> None:
+    _dev(x, "x"); _dev(y, "y", x.dtype); _dev(scale, "scale", torch.float32)
+    if y.numel() != x.numel():
+        raise ValueError("y must have as many elements as x")
+    _check(load_library().sasq_fakequant_fwd(_ptr(x), _ptr(y), x.numel(), _dt(x), _ptr(scale), int(bits),
+                                             _stream(stream)), "sasq_fakequant_fwd")
+
+
+def sasq_fakequant_bwd_workspace(numel: int) -> int:
+    return int(load_library().sasq_fakequant_bwd_workspace(int(numel)))
+
+
+def sasq_fakequant_bwd(x, grad_y, grad_x, grad_scale, scale, workspace, bits: int = 8, accumulate: bool = False,
+                       stream=None) -> None:
+    _dev(x, "x"); _dev(grad_y, "grad_y", x.dtype); _dev(grad_x, "grad_x", x.dtype)
+    _dev(grad_scale, "grad_scale", torch.float32); _dev(scale, "scale", torch.float32); _dev(workspace, "workspace")
+    if grad_y.numel() != x.numel() or grad_x.numel() != x.numel():
+        raise ValueError("grad_y and grad_x must have as many elements as x")
+    _check(load_library().sasq_fakequant_bwd(_ptr(x), _ptr(grad_y), _ptr(grad_x), _ptr(grad_scale), int(bool(accumulate)),
+                                             x.numel(), _dt(x), _ptr(scale), int(bits), _ptr(workspace),
+                                             _nbytes(workspace), _stream(stream)), "sasq_fakequant_bwd")
+
+
+def sasq_fakequant_fwd_bwd(x, grad_y, y, grad_x, grad_scale, scale, workspace, bits: int = 8,
+                           accumulate: bool = False, stream=None) -> None:
+    _dev(x, "x"); _dev(grad_y, "grad_y", x.dtype); _dev(y, "y", x.dtype); _dev(grad_x, "grad_x", x.dtype)
+    _dev(grad_scale, "grad_scale", torch.float32); _dev(scale, "scale", torch.float32); _dev(workspace, "workspace")
+    if grad_y.numel() != x.numel() or grad_x.numel() != x.numel() or y.numel() != x.numel():
+        raise ValueError("grad_y, y and grad_x must have as many elements as x")
+    _check(load_library().sasq_fakequant_fwd_bwd(_ptr(x), _ptr(grad_y), _ptr(y), _ptr(grad_x), _ptr(grad_scale),
+                                                 int(bool(accumulate)), x.numel(), _dt(x), _ptr(scale), int(bits),
+                                                 _ptr(workspace), _nbytes(workspace), _stream(stream)),
+           "sasq_fakequant_fwd_bwd")
+
+
+def sasq_fakequant_multi_workspace(n_tensors: int) -> int:
+    return int(load_library().sasq_fakequant_multi_workspace(int(n_tensors)))
+
+
+def sasq_fakequant_fwd_bwd_multi(tensors, scales, grad_scales, workspace, bits: int = 8, accumulate: bool = False,
+                                 stream=None) -> None:
+    """tensors: sequence of (x, grad_y | None, y | None, grad_x | None, scale_index)."""
+    n = len(tensors)
+    descs = (QDesc * max(n, 1))()
+    dt = None
+    for i, (x, gy, y, gx, idx) in enumerate(tensors):
+        _dev(x, "x")
+        for name, t in (("grad_y", gy), ("y", y), ("grad_x", gx)):
+            if t is not None:
+                _dev(t, name, x.dtype)
+                if t.numel() != x.numel():
+                    raise ValueError(f"{name} must have as many elements as x")
+        if dt is None:
+            dt = _dt(x)
+        elif dt != _dt(x):
+            raise TypeError("all tensors of one call must share a dtype")
+        descs[i] = QDesc(_ptr(x), _ptr(gy), _ptr(y), _ptr(gx), x.numel(), int(idx), 0)
+    _dev(scales, "scales", torch.float32)
+    if grad_scales is not None:
+        _dev(grad_scales, "grad_scales", torch.float32)
+    if workspace is not None:
+        _dev(workspace, "workspace")
+    _check(load_library().sasq_fakequant_fwd_bwd_multi(descs, n, _ptr(scales), _ptr(grad_scales), scales.numel(),
+                                                       int(bool(accumulate)), SASQ_BF16 if dt is None else dt,
+                                                       int(bits), _ptr(workspace), _nbytes(workspace),
+                                                       _stream(stream)), "sasq_fakequant_fwd_bwd_multi")
+
+
+def sasq_static_w8a8_linear_workspace(T: int, N: int, K: int) -> int:
+    return int(load_library().sasq_static_w8a8_linear_workspace(int(T), int(N), int(K)))
+
+
+def sasq_static_w8a8_linear(x, w, w_scale, x_scale, y, bias=None, acc_out=None, workspace=None, bits: int = 8,
+                            stream=None) -> None:
+    """x [T, K] fp16/bf16, w [N, K] int8, w_scale [N] fp32, x_scale [1] fp32, y [T, N]."""
+    _dev(x, "x"); _dev(w, "w", torch.int8); _dev(w_scale, "w_scale", torch.float32)
+    _dev(x_scale, "x_scale", torch.float32); _dev(y, "y", x.dtype)
+    if bias is not None:
+        _dev(bias, "bias", x.dtype)
+    if acc_out is not None:
+        _dev(acc_out, "acc_out", torch.int32)
+    if workspace is not None:
+        _dev(workspace, "workspace")
+    if x.dim() != 2 or w.dim() != 2 or x.shape[1] != w.shape[1]:
+        raise ValueError("x must be [T, K] and w [N, K]")
+    T, K = x.shape
+    N = w.shape[0]
+    if tuple(y.shape) != (T, N) or w_scale.numel() != N or (bias is not None and bias.numel() != N):
+        raise ValueError("y must be [T, N], w_scale and bias [N]")
+    if acc_out is not None and tuple(acc_out.shape) != (T, N):
+        raise ValueError("acc_out must be [T, N]")
+    _check(load_library().sasq_static_w8a8_linear(_ptr(x), _ptr(w), _ptr(w_scale), _ptr(x_scale), _ptr(bias), _ptr(y),
+                                                  _ptr(acc_out), T, N, K, _dt(x), int(bits), _ptr(workspace),
+                                                  _nbytes(workspace), _stream(stream)), "sasq_static_w8a8_linear")
+
+
+def sasq_device_status(stream=None) -> int:
+    """Synchronises the stream; returns and clears the sticky device status (0 = OK)."""
+    return int(load_library().sasq_device_status(_stream(stream)))

@@ -1,0 +1,195 @@
+// C-ABI entry points of the fake-quant forward / backward / fused path.
+#include "fakequant_kernels.cuh"
+
+namespace sasq {
+
+SASQ_DEFINE_STATUS_WORD(g_fakequant_status)
+
+int fakequant_status_read_and_clear(cudaStream_t st) { return g_fakequant_status_read_and_clear(st); }
+
+namespace {
+
+// launch shape of the streaming kernel
+constexpr int kThreads = 256;
+constexpr int kUnroll = 2;
+constexpr int kBlocksPerSM = 4;
+constexpr int kLoadHint = 1;
+constexpr int kStoreHint = 1;
+
+int* status_word_ptr() {
+    int* p = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_fakequant_status) != cudaSuccess) return nullptr;
+    return p;
+}
+
+template <bool BF, bool FWD, bool BWD>
+cudaError_t launch_stream(const QParams& p, int grid, cudaStream_t st) {
+    fakequant_kernel<BF, FWD, BWD, kThreads, kUnroll, kBlocksPerSM, kLoadHint, kStoreHint>
+        <<<grid, kThreads, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+template <bool BF>
+cudaError_t launch_mode(bool fwd, bool bwd, const QParams& p, int grid, cudaStream_t st) {
+    if (fwd && bwd) return launch_stream<BF, true, true>(p, grid, st);
+    if (fwd) return launch_stream<BF, true, false>(p, grid, st);
+    return launch_stream<BF, false, true>(p, grid, st);
+}
+
+int grid_for(long long max_numel, int sm_count) {
+    long long g = (long long)sm_count * kBlocksPerSM;
+    const long long need = ((max_numel >> 3) + kThreads - 1) / kThreads;
+    if (g > need) g = need;
+    if (g > kMaxGrid) g = kMaxGrid;
+    if (g < 1) g = 1;
+    return (int)g;
+}
+
+int run_multi(const sasq_qdesc_t* descs, int n_tensors, const float* scales_dev, float* grad_scales_dev,
+              int n_scales, int accumulate, int dt, int bits, void* workspace, size_t ws_bytes, void* stream) {
+    if (n_tensors < 0 || n_scales <= 0 || (n_tensors > 0 && descs == nullptr)) return SASQ_ERR_INVALID_ARG;
+    if (scales_dev == nullptr) return SASQ_ERR_INVALID_ARG;
+    if (bits < 2 || bits > 8) return SASQ_ERR_INVALID_ARG;
+    if (dt != SASQ_F16 && dt != SASQ_BF16) return SASQ_ERR_INVALID_ARG;
+    if (n_tensors == 0) return SASQ_OK;
+
+    const bool fwd = descs[0].y != nullptr;
+    const bool bwd = descs[0].grad_y != nullptr;
+    long long max_numel = 0;
+    for (int i = 0; i < n_tensors; ++i) {
+        const sasq_qdesc_t& d = descs[i];
+        if (d.numel < 0 || d.reserved != 0) return SASQ_ERR_INVALID_ARG;
+        if (d.scale_index < 0 || d.scale_index >= n_scales) return SASQ_ERR_INVALID_ARG;
+        if ((d.y != nullptr) != fwd || (d.grad_y != nullptr) != bwd) return SASQ_ERR_INVALID_ARG;
+        if ((d.grad_y != nullptr) != (d.grad_x != nullptr)) return SASQ_ERR_INVALID_ARG;
+        if (d.numel > 0 && d.x == nullptr) return SASQ_ERR_INVALID_ARG;
+        if (!aligned16(d.x) || !aligned16(d.y) || !aligned16(d.grad_y) || !aligned16(d.grad_x))
+            return SASQ_ERR_INVALID_ARG;
+        if (d.numel > max_numel) max_numel = d.numel;
+    }
+    if (!fwd && !bwd) return SASQ_ERR_INVALID_ARG;
+    if (bwd) {
+        if (grad_scales_dev == nullptr) return SASQ_ERR_INVALID_ARG;
+        if (workspace == nullptr || !aligned16(workspace) ||
+            ws_bytes < sasq_fakequant_multi_workspace(n_tensors))
+            return SASQ_ERR_WORKSPACE;
+    }
+    const int sm_count = device_sm_count_if_sm100();
+    if (sm_count <= 0) return SASQ_ERR_UNSUPPORTED;
+    int* status = status_word_ptr();
+    if (status == nullptr) return SASQ_ERR_CUDA;
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int grid = grid_for(max_numel, sm_count);
+    // slots already written by an earlier chunk of this call are added to afterwards
+    // (only possible when n_tensors > kMaxDescsPerLaunch)
+    for (int base = 0; base < n_tensors; base += kMaxDescsPerLaunch) {
+        const int n = (n_tensors - base < kMaxDescsPerLaunch) ? (n_tensors - base) : kMaxDescsPerLaunch;
+        QParams p{};
+        CombineParams c{};
+        for (int i = 0; i < n; ++i) {
+            const sasq_qdesc_t& d = descs[base + i];
+            p.d[i].x = static_cast<const uint4*>(d.x);
+            p.d[i].g = static_cast<const uint4*>(d.grad_y);
+            p.d[i].y = static_cast<uint4*>(d.y);
+            p.d[i].dx = static_cast<uint4*>(d.grad_x);
+            p.d[i].numel = d.numel;
+            p.d[i].scale_index = d.scale_index;
+            c.scale_index[i] = d.scale_index;
+            bool seen_before = false;
+            for (int k = 0; k < base && !seen_before; ++k) seen_before = (descs[k].scale_index == d.scale_index);
+            if (accumulate || seen_before) c.accumulate_mask |= (1u << i);
+        }
+        p.n = n;
+        p.scales = scales_dev;
+        p.partials = static_cast<double*>(workspace) + (size_t)base * kMaxGrid;
+        p.qn = (float)(1 << (bits - 1));
+        p.qp = (float)((1 << (bits - 1)) - 1);
+        p.status = status;
+        cudaError_t e = (dt == SASQ_BF16) ? launch_mode<true>(fwd, bwd, p, grid, st)
+                                          : launch_mode<false>(fwd, bwd, p, grid, st);
+        if (e != cudaSuccess) return SASQ_ERR_CUDA;
+        if (bwd) {
+            c.n = n;
+            c.grid = grid;
+            c.partials = p.partials;
+            c.grad_scales = grad_scales_dev;
+            fakequant_combine_kernel<<<n, kCombineThreads, 0, st>>>(c);
+            if (cudaGetLastError() != cudaSuccess) return SASQ_ERR_CUDA;
+        }
+    }
+    return SASQ_OK;
+}
+
+int run_single(const void* x, const void* grad_y, void* y, void* grad_x, float* grad_scale_dev, int accumulate,
+               int64_t numel, int dt, const float* scale_dev, int bits, void* workspace, size_t ws_bytes,
+               void* stream, bool fwd, bool bwd) {
+    if (numel < 0) return SASQ_ERR_INVALID_ARG;
+    if (scale_dev == nullptr) return SASQ_ERR_INVALID_ARG;
+    if (bits < 2 || bits > 8) return SASQ_ERR_INVALID_ARG;
+    if (dt != SASQ_F16 && dt != SASQ_BF16) return SASQ_ERR_INVALID_ARG;
+    if (bwd && grad_scale_dev == nullptr) return SASQ_ERR_INVALID_ARG;
+    if (numel > 0) {
+        if (x == nullptr || (fwd && y == nullptr) || (bwd && (grad_y == nullptr || grad_x == nullptr)))
+            return SASQ_ERR_INVALID_ARG;
+    }
+    if (numel == 0) {
+        if (bwd && !accumulate) {
+            if (cudaMemsetAsync(grad_scale_dev, 0, sizeof(float), static_cast<cudaStream_t>(stream)) != cudaSuccess)
+                return SASQ_ERR_CUDA;
+        }
+        return SASQ_OK;
+    }
+    sasq_qdesc_t d{};
+    d.x = x;
+    d.grad_y = bwd ? grad_y : nullptr;
+    d.y = fwd ? y : nullptr;
+    d.grad_x = bwd ? grad_x : nullptr;
+    d.numel = numel;
+    d.scale_index = 0;
+    return run_multi(&d, 1, scale_dev, grad_scale_dev, 1, accumulate, dt, bits, workspace, ws_bytes, stream);
+}
+
+}  // namespace
+}  // namespace sasq
+
+extern "C" {
+
+size_t sasq_fakequant_bwd_workspace(int64_t numel) {
+    (void)numel;
+    return sasq_fakequant_multi_workspace(1);
+}
+
+size_t sasq_fakequant_multi_workspace(int n_tensors) {
+    if (n_tensors < 1) n_tensors = 1;
+    return (size_t)n_tensors * sasq::kMaxGrid * sizeof(double);
+}
+
+int sasq_fakequant_fwd(const void* x, void* y, int64_t numel, int dt, const float* scale_dev, int bits,
+                       void* stream) {
+    return sasq::run_single(x, nullptr, y, nullptr, nullptr, 0, numel, dt, scale_dev, bits, nullptr, 0, stream,
+                            true, false);
+}
+
+int sasq_fakequant_bwd(const void* x, const void* grad_y, void* grad_x, float* grad_scale_dev, int accumulate,
+                       int64_t numel, int dt, const float* scale_dev, int bits, void* workspace, size_t ws_bytes,
+                       void* stream) {
+    return sasq::run_single(x, grad_y, nullptr, grad_x, grad_scale_dev, accumulate, numel, dt, scale_dev, bits,
+                            workspace, ws_bytes, stream, false, true);
+}
+
+int sasq_fakequant_fwd_bwd(const void* x, const void* grad_y, void* y, void* grad_x, float* grad_scale_dev,
+                           int accumulate, int64_t numel, int dt, const float* scale_dev, int bits,
+                           void* workspace, size_t ws_bytes, void* stream) {
+    return sasq::run_single(x, grad_y, y, grad_x, grad_scale_dev, accumulate, numel, dt, scale_dev, bits,
+                            workspace, ws_bytes, stream, true, true);
+}
+
+int sasq_fakequant_fwd_bwd_multi(const sasq_qdesc_t* descs_host, int n_tensors, const float* scales_dev,
+                                 float* grad_scales_dev, int n_scales, int accumulate, int dt, int bits,
+                                 void* workspace, size_t ws_bytes, void* stream) {
+    return sasq::run_multi(descs_host, n_tensors, scales_dev, grad_scales_dev, n_scales, accumulate, dt, bits,
+                           workspace, ws_bytes, stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,222 @@
+// Fake-quant forward / STE backward / fused kernels (sm_100a).
+//
+// One streaming pass over the tensors: 128-bit coalesced loads of x (and the
+// upstream gradient), fp32 arithmetic in the fixed order
+//     t = x * fl32(1/s);  r = rint(t);  c = clamp(r, -Qn, Qp)          (Eq. 1)
+//     y = narrow(c * s)                                                (Sec. 4.2)
+//     m = (c == r);  dx = m ? g : 0                                    (Eq. 4)
+//     ds += g * (m ? r - t : c)                                        (chain rule)
+// 128-bit stores of y and dx, and a deterministic reduction of ds:
+// fp32 tree over the 8 products of a vector -> double per thread -> warp
+// shuffles -> shared memory -> one double per (tensor, block) in the workspace.
+// A second tiny kernel adds the block partials in a fixed order.
+//
+// The path is HBM-bound: 4 B / element forward, 6 B backward, 8 B fused.
+#pragma once
+
+#include "common.cuh"
+
+namespace sasq {
+
+constexpr int kMaxDescsPerLaunch = 32;   // descriptors that fit one launch's parameter block
+constexpr int kMaxGrid = 2048;           // upper bound on blocks per launch (sizes the workspace)
+
+struct QDesc {
+    const uint4* x;
+    const uint4* g;
+    uint4* y;
+    uint4* dx;
+    long long numel;
+    int scale_index;
+    int pad;
+};
+
+struct QParams {
+    QDesc d[kMaxDescsPerLaunch];
+    const float* scales;
+    double* partials;        // [n][gridDim.x]
+    int n;
+    float qn;                // 2^(b-1)
+    float qp;                // 2^(b-1) - 1
+    int* status;
+};
+
+struct Quant2 {
+    uint32_t y;      // two narrowed outputs
+    uint32_t dx;     // two masked gradients
+    float p0, p1;    // g * dy/ds
+};
+
+template <bool BF, bool FWD, bool BWD>
+__device__ __forceinline__ Quant2 quant_pair(uint32_t xw, uint32_t gw, float s, float inv, float qn, float qp) {
+    Quant2 o;
+    const float2 xf = widen2<BF>(xw);
+    const float t0 = __fmul_rn(xf.x, inv);
+    const float t1 = __fmul_rn(xf.y, inv);
+    const float r0 = rintf(t0);
+    const float r1 = rintf(t1);
+    const float c0 = fminf(fmaxf(r0, -qn), qp);
+    const float c1 = fminf(fmaxf(r1, -qn), qp);
+    if constexpr (FWD) {
+        o.y = narrow2<BF>(__fmul_rn(c0, s), __fmul_rn(c1, s));
+    }
+    if constexpr (BWD) {
+        const float2 gf = widen2<BF>(gw);
+        const bool in0 = (c0 == r0);      // false for NaN as well
+        const bool in1 = (c1 == r1);
+        o.dx = (in0 ? (gw & 0x0000FFFFu) : 0u) | (in1 ? (gw & 0xFFFF0000u) : 0u);
+        o.p0 = __fmul_rn(gf.x, in0 ? __fsub_rn(r0, t0) : c0);
+        o.p1 = __fmul_rn(gf.y, in1 ? __fsub_rn(r1, t1) : c1);
+    }
+    return o;
+}
+
+template <int HINT>
+__device__ __forceinline__ uint4 load16(const uint4* p) {
+    uint4 v;
+    if constexpr (HINT == 0) {
+        v = *p;
+    } else if constexpr (HINT == 1) {
+        asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    } else {
+        asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    }
+    return v;
+}
+
+template <int HINT>
+__device__ __forceinline__ void store16(uint4* p, const uint4& v) {
+    if constexpr (HINT == 0) {
+        *p = v;
+    } else {
+        asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                     : "memory");
+    }
+}
+
+// Block-level sum of one double per thread in a fixed order: lanes by xor
+// shuffles (16, 8, 4, 2, 1), then warp 0 adds the warp sums in warp order.
+template <int THREADS>
+__device__ __forceinline__ double block_sum_fixed(double v, double* smem /* [THREADS/32] */) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) smem[warp] = v;
+    __syncthreads();
+    double tot = 0.0;
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int w = 0; w < THREADS / 32; ++w) tot += smem[w];
+    }
+    __syncthreads();
+    return tot;   // valid in thread 0
+}
+
+template <bool BF, bool FWD, bool BWD, int THREADS, int UNROLL, int MIN_BLOCKS, int LHINT, int SHINT>
+__global__ void __launch_bounds__(THREADS, MIN_BLOCKS) fakequant_kernel(const __grid_constant__ QParams p) {
+    __shared__ double warp_sums[THREADS / 32];
+    const float qn = p.qn, qp = p.qp;
+    const long long gtid = (long long)blockIdx.x * THREADS + threadIdx.x;
+    const long long gstride = (long long)gridDim.x * THREADS;
+
+    for (int ti = 0; ti < p.n; ++ti) {
+        const QDesc& d = p.d[ti];
+        const float s = __ldg(p.scales + d.scale_index);
+        const float inv = __fdiv_rn(1.0f, s);
+        if (gtid == 0 && scale_is_bad(s)) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
+        const long long nvec = d.numel >> 3;
+        double acc = 0.0;
+
+        for (long long v0 = gtid; v0 < nvec; v0 += gstride * UNROLL) {
+            uint4 xv[UNROLL], gv[UNROLL];
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const long long v = v0 + (long long)u * gstride;
+                if (v < nvec) {
+                    xv[u] = load16<LHINT>(d.x + v);
+                    if constexpr (BWD) gv[u] = load16<LHINT>(d.g + v);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const long long v = v0 + (long long)u * gstride;
+                if (v < nvec) {
+                    const uint32_t xw[4] = {xv[u].x, xv[u].y, xv[u].z, xv[u].w};
+                    uint32_t gw[4] = {0u, 0u, 0u, 0u};
+                    if constexpr (BWD) { gw[0] = gv[u].x; gw[1] = gv[u].y; gw[2] = gv[u].z; gw[3] = gv[u].w; }
+                    Quant2 q[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) q[j] = quant_pair<BF, FWD, BWD>(xw[j], gw[j], s, inv, qn, qp);
+                    if constexpr (FWD) store16<SHINT>(d.y + v, make_uint4(q[0].y, q[1].y, q[2].y, q[3].y));
+                    if constexpr (BWD) {
+                        store16<SHINT>(d.dx + v, make_uint4(q[0].dx, q[1].dx, q[2].dx, q[3].dx));
+                        const float a = __fadd_rn(__fadd_rn(q[0].p0, q[0].p1), __fadd_rn(q[1].p0, q[1].p1));
+                        const float b = __fadd_rn(__fadd_rn(q[2].p0, q[2].p1), __fadd_rn(q[3].p0, q[3].p1));
+                        acc += (double)__fadd_rn(a, b);
+                    }
+                }
+            }
+        }
+
+        // ragged tail (numel % 8 elements): one element per thread of the last block
+        const int tail = (int)(d.numel & 7);
+        if (tail != 0 && blockIdx.x == gridDim.x - 1 && threadIdx.x < tail) {
+            const long long i = (nvec << 3) + threadIdx.x;
+            const uint16_t xh = reinterpret_cast<const uint16_t*>(d.x)[i];
+            const float xf = widen1<BF>(xh);
+            const float t = __fmul_rn(xf, inv);
+            const float r = rintf(t);
+            const float c = fminf(fmaxf(r, -qn), qp);
+            if constexpr (FWD) reinterpret_cast<uint16_t*>(d.y)[i] = narrow1<BF>(__fmul_rn(c, s));
+            if constexpr (BWD) {
+                const uint16_t gh = reinterpret_cast<const uint16_t*>(d.g)[i];
+                const bool in = (c == r);
+                reinterpret_cast<uint16_t*>(d.dx)[i] = in ? gh : (uint16_t)0;
+                acc += (double)__fmul_rn(widen1<BF>(gh), in ? __fsub_rn(r, t) : c);
+            }
+        }
+
+        if constexpr (BWD) {
+            const double tot = block_sum_fixed<THREADS>(acc, warp_sums);
+            if (threadIdx.x == 0) p.partials[(long long)ti * gridDim.x + blockIdx.x] = tot;
+        }
+    }
+}
+
+// Second stage: block j acts iff descriptor j is the first of its factor slot in
+// this launch; it adds the partials of every descriptor of that slot, in
+// descriptor order then block order, and writes (or adds to) grad_scales[slot].
+struct CombineParams {
+    int scale_index[kMaxDescsPerLaunch];
+    int n;
+    int grid;                 // partials per descriptor
+    unsigned accumulate_mask; // bit j: descriptor j's slot is added to, not overwritten
+    const double* partials;
+    float* grad_scales;
+};
+
+constexpr int kCombineThreads = 256;
+
+__global__ void __launch_bounds__(kCombineThreads) fakequant_combine_kernel(const __grid_constant__ CombineParams p) {
+    __shared__ double warp_sums[kCombineThreads / 32];
+    const int j = blockIdx.x;
+    const int slot = p.scale_index[j];
+    if (slot < 0) return;                                   // descriptor without a backward part
+    for (int k = 0; k < j; ++k)
+        if (p.scale_index[k] == slot) return;               // not the first of its slot
+    double acc = 0.0;
+    for (int k = j; k < p.n; ++k) {
+        if (p.scale_index[k] != slot) continue;
+        const double* part = p.partials + (long long)k * p.grid;
+        for (int i = threadIdx.x; i < p.grid; i += kCombineThreads) acc += part[i];
+    }
+    const double tot = block_sum_fixed<kCombineThreads>(acc, warp_sums);
+    if (threadIdx.x == 0) {
+        const float prev = ((p.accumulate_mask >> j) & 1u) ? p.grad_scales[slot] : 0.0f;
+        p.grad_scales[slot] = prev + (float)tot;
+    }
+}
+
+}  // namespace sasq
