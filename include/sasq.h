@@ -144,6 +144,26 @@ SASQ_API int sasq_static_w8a8_linear(const void* x, const int8_t* w, const float
                             const void* bias, void* y, int32_t* acc_out, int64_t T, int64_t N, int64_t K,
                             int dt, int bits, void* workspace, size_t ws_bytes, void* stream);
 
+/* ---- PTQ initialisation (Sec. 4.1), set-up only, not on the hot path ---- */
+
+/* Bytes of scratch sasq_absmax_scale needs. */
+SASQ_API size_t sasq_absmax_scale_workspace(int64_t numel);
+
+/* Max-based factor of one calibration batch (Eq. 1): scale_out_dev[0] =
+ * max_i |x[i]| / Qp in fp32.  The paper initialises each factor with the average
+ * of these values over the calibration batches; the caller averages.  x:
+ * [numel] of `dt`; an all-zero or empty x gives 0 (not a usable factor). */
+SASQ_API int sasq_absmax_scale(const void* x, int64_t numel, int dt, int bits, float* scale_out_dev, void* workspace,
+                               size_t ws_bytes, void* stream);
+
+/* Per-output-channel symmetric weight quantizer (Eq. 1 applied to each column of
+ * the paper's K x N weight, i.e. each row of w[N, K]; weights are always
+ * quantized per channel, Sec. 5.1):  w_scale[n] = max_k |w[n,k]| / Qp (1 for an
+ * all-zero row), w_int[n,k] = clamp(rint(w[n,k] * fl32(1 / w_scale[n])), -Qn, Qp).
+ * w: [N, K] fp32; w_int: [N, K] int8; w_scale: [N] fp32. */
+SASQ_API int sasq_quantize_weight(const float* w, int8_t* w_int, float* w_scale, int64_t N, int64_t K, int bits,
+                                  void* stream);
+
 /* Synchronises `stream`, returns the sticky device status word of the current
  * device (SASQ_OK, SASQ_ERR_BAD_SCALE or SASQ_ERR_TIMEOUT) and clears it. */
 SASQ_API int sasq_device_status(void* stream);

@@ -17,11 +17,14 @@ __all__ = [
     "SasqError", "SASQ_F16", "SASQ_BF16", "library_path", "load_library", "sasq_status_string",
     "sasq_fakequant_fwd", "sasq_fakequant_bwd_workspace", "sasq_fakequant_bwd", "sasq_fakequant_fwd_bwd",
     "sasq_fakequant_multi_workspace", "sasq_fakequant_fwd_bwd_multi", "sasq_static_w8a8_linear_workspace",
-    "sasq_static_w8a8_linear", "sasq_device_status", "QDesc",
+    "sasq_static_w8a8_linear", "sasq_device_status", "QDesc", "sasq_absmax_scale_workspace", "sasq_absmax_scale",
+    "sasq_quantize_weight", "LAUNCHES_PER_LINEAR",
 ]
 
 SASQ_F16 = 0
 SASQ_BF16 = 1
+# kernels one sasq_static_w8a8_linear call launches (activation quantizer + GEMM); used to count launches
+LAUNCHES_PER_LINEAR = 2
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libsasq_b200.so")
@@ -75,6 +78,12 @@ def load_library() -> ctypes.CDLL:
     L.sasq_static_w8a8_linear.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, sz, vp]
     L.sasq_device_status.restype = i32
     L.sasq_device_status.argtypes = [vp]
+    L.sasq_absmax_scale_workspace.restype = sz
+    L.sasq_absmax_scale_workspace.argtypes = [i64]
+    L.sasq_absmax_scale.restype = i32
+    L.sasq_absmax_scale.argtypes = [vp, i64, i32, i32, vp, vp, sz, vp]
+    L.sasq_quantize_weight.restype = i32
+    L.sasq_quantize_weight.argtypes = [vp, vp, vp, i64, i64, i32, vp]
     _lib = L
     return L
 
@@ -226,3 +235,23 @@ def sasq_static_w8a8_linear(x, w, w_scale, x_scale, y, bias=None, acc_out=None, 
 def sasq_device_status(stream=None) -> int:
     """Synchronises the stream; returns and clears the sticky device status (0 = OK)."""
     return int(load_library().sasq_device_status(_stream(stream)))
+
+
+def sasq_absmax_scale_workspace(numel: int) -> int:
+    return int(load_library().sasq_absmax_scale_workspace(int(numel)))
+
+
+def sasq_absmax_scale(x, scale_out, workspace, bits: int = 8, stream=None) -> None:
+    """scale_out[0] = max|x| / Qp (Eq. 1) of one calibration batch."""
+    _dev(x, "x"); _dev(scale_out, "scale_out", torch.float32); _dev(workspace, "workspace")
+    _check(load_library().sasq_absmax_scale(_ptr(x), x.numel(), _dt(x), int(bits), _ptr(scale_out), _ptr(workspace),
+                                            _nbytes(workspace), _stream(stream)), "sasq_absmax_scale")
+
+
+def sasq_quantize_weight(w, w_int, w_scale, bits: int = 8, stream=None) -> None:
+    """w [N, K] fp32 -> w_int [N, K] int8 and w_scale [N] fp32, one factor per output channel."""
+    _dev(w, "w", torch.float32); _dev(w_int, "w_int", torch.int8); _dev(w_scale, "w_scale", torch.float32)
+    if w.dim() != 2 or tuple(w_int.shape) != tuple(w.shape) or w_scale.numel() != w.shape[0]:
+        raise ValueError("w and w_int must be [N, K], w_scale [N]")
+    _check(load_library().sasq_quantize_weight(_ptr(w), _ptr(w_int), _ptr(w_scale), w.shape[0], w.shape[1], int(bits),
+                                               _stream(stream)), "sasq_quantize_weight")

@@ -1,0 +1,133 @@
+// PTQ initialisation helpers (Sec. 4.1; Eq. 1): the max-based activation factor
+// S = max|X| / Qp of one calibration batch, and the per-output-channel weight
+// quantizer.  They run once at set-up, not on the hot path.
+#include "common.cuh"
+
+namespace sasq {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kMaxBlocks = 1024;
+
+__device__ __forceinline__ float block_max(float v, float* smem) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, off));
+    if ((threadIdx.x & 31) == 0) smem[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float m = 0.0f;
+    if (threadIdx.x < 32) {
+        m = (threadIdx.x < kThreads / 32) ? smem[threadIdx.x] : 0.0f;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, off));
+    }
+    __syncthreads();
+    return m;   // valid in warp 0
+}
+
+template <bool BF>
+__global__ void __launch_bounds__(kThreads) absmax_partial_kernel(const uint16_t* __restrict__ x, long long numel,
+                                                                  float* __restrict__ partial) {
+    __shared__ float smem[kThreads / 32];
+    float m = 0.0f;
+    const long long stride = (long long)gridDim.x * kThreads;
+    const long long nvec = numel >> 3;
+    const uint4* xv = reinterpret_cast<const uint4*>(x);
+    for (long long i = (long long)blockIdx.x * kThreads + threadIdx.x; i < nvec; i += stride) {
+        const uint4 v = xv[i];
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float2 f = widen2<BF>(w[j]);
+            m = fmaxf(m, fmaxf(fabsf(f.x), fabsf(f.y)));
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x < (int)(numel & 7))
+        m = fmaxf(m, fabsf(widen1<BF>(x[(nvec << 3) + threadIdx.x])));
+    m = block_max(m, smem);
+    if (threadIdx.x == 0) partial[blockIdx.x] = m;
+}
+
+__global__ void __launch_bounds__(kThreads) absmax_final_kernel(const float* __restrict__ partial, int n, float qp,
+                                                                float* __restrict__ scale_out) {
+    __shared__ float smem[kThreads / 32];
+    float m = 0.0f;
+    for (int i = threadIdx.x; i < n; i += kThreads) m = fmaxf(m, partial[i]);
+    m = block_max(m, smem);
+    if (threadIdx.x == 0) scale_out[0] = __fdiv_rn(m, qp);
+}
+
+// one block per output channel (row of w[N, K])
+__global__ void __launch_bounds__(kThreads) quantize_weight_kernel(const float* __restrict__ w, int8_t* __restrict__ w_int,
+                                                                   float* __restrict__ w_scale, long long K, float qn,
+                                                                   float qp) {
+    __shared__ float smem[kThreads / 32];
+    __shared__ float s_inv;
+    const float* row = w + (long long)blockIdx.x * K;
+    float m = 0.0f;
+    for (long long k = threadIdx.x; k < K; k += kThreads) m = fmaxf(m, fabsf(row[k]));
+    m = block_max(m, smem);
+    if (threadIdx.x == 0) {
+        const float sc = m > 0.0f ? __fdiv_rn(m, qp) : 1.0f;
+        w_scale[blockIdx.x] = sc;
+        s_inv = __fdiv_rn(1.0f, sc);
+    }
+    __syncthreads();
+    const float inv = s_inv;
+    int8_t* out = w_int + (long long)blockIdx.x * K;
+    for (long long k = threadIdx.x; k < K; k += kThreads) {
+        const float r = rintf(__fmul_rn(row[k], inv));
+        out[k] = (int8_t)(int)fminf(fmaxf(r, -qn), qp);
+    }
+}
+
+}  // namespace
+}  // namespace sasq
+
+extern "C" {
+
+size_t sasq_absmax_scale_workspace(int64_t numel) {
+    (void)numel;
+    return (size_t)sasq::kMaxBlocks * sizeof(float);
+}
+
+int sasq_absmax_scale(const void* x, int64_t numel, int dt, int bits, float* scale_out_dev, void* workspace,
+                      size_t ws_bytes, void* stream) {
+    using namespace sasq;
+    if (numel < 0 || scale_out_dev == nullptr || bits < 2 || bits > 8) return SASQ_ERR_INVALID_ARG;
+    if (dt != SASQ_F16 && dt != SASQ_BF16) return SASQ_ERR_INVALID_ARG;
+    if (numel > 0 && (x == nullptr || !aligned16(x))) return SASQ_ERR_INVALID_ARG;
+    if (workspace == nullptr || !aligned16(workspace) || ws_bytes < sasq_absmax_scale_workspace(numel))
+        return SASQ_ERR_WORKSPACE;
+    const int sm_count = device_sm_count_if_sm100();
+    if (sm_count <= 0) return SASQ_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    long long blocks = ((numel >> 3) + kThreads - 1) / kThreads;
+    if (blocks < 1) blocks = 1;
+    if (blocks > kMaxBlocks) blocks = kMaxBlocks;
+    if (blocks > (long long)sm_count * 4) blocks = (long long)sm_count * 4;
+    float* partial = static_cast<float*>(workspace);
+    if (dt == SASQ_BF16)
+        absmax_partial_kernel<true><<<(int)blocks, kThreads, 0, st>>>(static_cast<const uint16_t*>(x), numel, partial);
+    else
+        absmax_partial_kernel<false><<<(int)blocks, kThreads, 0, st>>>(static_cast<const uint16_t*>(x), numel, partial);
+    if (cudaGetLastError() != cudaSuccess) return SASQ_ERR_CUDA;
+    absmax_final_kernel<<<1, kThreads, 0, st>>>(partial, (int)blocks, (float)((1 << (bits - 1)) - 1), scale_out_dev);
+    if (cudaGetLastError() != cudaSuccess) return SASQ_ERR_CUDA;
+    return SASQ_OK;
+}
+
+int sasq_quantize_weight(const float* w, int8_t* w_int, float* w_scale, int64_t N, int64_t K, int bits,
+                         void* stream) {
+    using namespace sasq;
+    if (N < 0 || K <= 0 || bits < 2 || bits > 8) return SASQ_ERR_INVALID_ARG;
+    if (N > 0 && (w == nullptr || w_int == nullptr || w_scale == nullptr)) return SASQ_ERR_INVALID_ARG;
+    if (N > 0x7FFFFFFF) return SASQ_ERR_UNSUPPORTED;
+    if (N == 0) return SASQ_OK;
+    if (device_sm_count_if_sm100() <= 0) return SASQ_ERR_UNSUPPORTED;
+    quantize_weight_kernel<<<(int)N, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        w, w_int, w_scale, K, (float)(1 << (bits - 1)), (float)((1 << (bits - 1)) - 1));
+    if (cudaGetLastError() != cudaSuccess) return SASQ_ERR_CUDA;
+    return SASQ_OK;
+}
+
+}  // extern "C"
