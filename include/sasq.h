@@ -111,6 +111,29 @@ SASQ_API int sasq_fakequant_fwd_bwd(const void* x, const void* grad_y, void* y, 
                            int accumulate, int64_t numel, int dt, const float* scale_dev, int bits,
                            void* workspace, size_t ws_bytes, void* stream);
 
+/* The same fused pass for callers that can neither allocate device memory nor
+ * hand over a workspace: for instance a plugin hook of an inference runtime that
+ * forbids allocation inside its execute call, or a process whose device memory
+ * is entirely owned by another allocator, so that a cudaMalloc here would fail
+ * or break its budget.  (The paper has no counterpart; this is a deployment
+ * convenience of the library.)  The block partials of the scale-gradient
+ * reduction live in a fixed 8 KiB array inside the library's device image, which
+ * every GPU that loads the library holds until the process exits.  The call
+ * itself performs no allocation of any kind.
+ *   - Results are identical, bit for bit, to sasq_fakequant_fwd_bwd.
+ *   - numel may be at most 2^30; larger tensors (or a device with more thread
+ *     blocks than the array has slots) give SASQ_ERR_UNSUPPORTED and no launch.
+ *   - The first call on each device looks up the array's device address (with
+ *     that device current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Its previous contents never
+ *     matter (every slot that is read is written first, nothing needs zeroing),
+ *     but two calls that overlap on the GPU -- different streams, or different
+ *     host threads without ordering -- race on it and corrupt each other's
+ *     grad_scale.  Order them on one stream or with events. */
+SASQ_API int sasq_fakequant_fwd_bwd_static(const void* x, const void* grad_y, void* y, void* grad_x,
+                                           float* grad_scale_dev, int accumulate, int64_t numel, int dt,
+                                           const float* scale_dev, int bits, void* stream);
+
 /* Bytes of scratch for a multi-tensor call with n_tensors descriptors. */
 SASQ_API size_t sasq_fakequant_multi_workspace(int n_tensors);
 

@@ -18,7 +18,7 @@ __all__ = [
     "sasq_fakequant_fwd", "sasq_fakequant_bwd_workspace", "sasq_fakequant_bwd", "sasq_fakequant_fwd_bwd",
     "sasq_fakequant_multi_workspace", "sasq_fakequant_fwd_bwd_multi", "sasq_static_w8a8_linear_workspace",
     "sasq_static_w8a8_linear", "sasq_device_status", "QDesc", "sasq_absmax_scale_workspace", "sasq_absmax_scale",
-    "sasq_quantize_weight", "LAUNCHES_PER_LINEAR",
+    "sasq_quantize_weight", "LAUNCHES_PER_LINEAR", "sasq_fakequant_fwd_bwd_static",
 ]
 
 SASQ_F16 = 0
@@ -68,6 +68,8 @@ def load_library() -> ctypes.CDLL:
     L.sasq_fakequant_bwd.argtypes = [vp, vp, vp, vp, i32, i64, i32, vp, i32, vp, sz, vp]
     L.sasq_fakequant_fwd_bwd.restype = i32
     L.sasq_fakequant_fwd_bwd.argtypes = [vp, vp, vp, vp, vp, i32, i64, i32, vp, i32, vp, sz, vp]
+    L.sasq_fakequant_fwd_bwd_static.restype = i32
+    L.sasq_fakequant_fwd_bwd_static.argtypes = [vp, vp, vp, vp, vp, i32, i64, i32, vp, i32, vp]
     L.sasq_fakequant_multi_workspace.restype = sz
     L.sasq_fakequant_multi_workspace.argtypes = [i32]
     L.sasq_fakequant_fwd_bwd_multi.restype = i32
@@ -255,3 +257,18 @@ def sasq_quantize_weight(w, w_int, w_scale, bits: int = 8, stream=None) -> None:
         raise ValueError("w and w_int must be [N, K], w_scale [N]")
     _check(load_library().sasq_quantize_weight(_ptr(w), _ptr(w_int), _ptr(w_scale), w.shape[0], w.shape[1], int(bits),
                                                _stream(stream)), "sasq_quantize_weight")
+
+
+def sasq_fakequant_fwd_bwd_static(x, grad_y, y, grad_x, grad_scale, scale, bits: int = 8, accumulate: bool = False,
+                                  stream=None) -> None:
+    """Fused forward + backward without any workspace argument: the reduction scratch is a fixed array inside the
+    library, for callers that are not allowed to allocate (see include/sasq.h).  Calls on one device must not
+    overlap; the first call on a device should be made outside stream capture."""
+    _dev(x, "x"); _dev(grad_y, "grad_y", x.dtype); _dev(y, "y", x.dtype); _dev(grad_x, "grad_x", x.dtype)
+    _dev(grad_scale, "grad_scale", torch.float32); _dev(scale, "scale", torch.float32)
+    if grad_y.numel() != x.numel() or grad_x.numel() != x.numel() or y.numel() != x.numel():
+        raise ValueError("grad_y, y and grad_x must have as many elements as x")
+    _check(load_library().sasq_fakequant_fwd_bwd_static(_ptr(x), _ptr(grad_y), _ptr(y), _ptr(grad_x),
+                                                        _ptr(grad_scale), int(bool(accumulate)), x.numel(), _dt(x),
+                                                        _ptr(scale), int(bits), _stream(stream)),
+           "sasq_fakequant_fwd_bwd_static")

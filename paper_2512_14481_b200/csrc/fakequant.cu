@@ -150,10 +150,90 @@ int run_single(const void* x, const void* grad_y, void* y, void* grad_x, float* 
     return run_multi(&d, 1, scale_dev, grad_scale_dev, 1, accumulate, dt, bits, workspace, ws_bytes, stream);
 }
 
+// ---------------------------------------------------------------------------
+// Variant for callers that cannot allocate: the block partials live in a
+// file-scope device array instead of a caller-provided workspace.
+// ---------------------------------------------------------------------------
+constexpr int kStaticPartials = 1024;                      // doubles: 8 KiB held by every device that loads the library
+constexpr int64_t kStaticMaxNumel = (int64_t)1 << 30;      // largest tensor the static-scratch call accepts
+static __device__ __align__(256) double g_static_partials[kStaticPartials];
+
+// Device address of the static scratch on the current device.  In host code the
+// array's name is only a handle; the address a kernel can use comes from the
+// runtime, once per device, with that device current.
+double* static_partials_ptr(int* err) {
+    static double* cache[64] = {nullptr};
+    *err = SASQ_OK;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { *err = SASQ_ERR_CUDA; return nullptr; }
+    if (cache[dev] == nullptr) {
+        double* p = nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_partials) != cudaSuccess || p == nullptr) {
+            *err = SASQ_ERR_CUDA;
+            return nullptr;
+        }
+        cache[dev] = p;
+    }
+    return cache[dev];
+}
+
 }  // namespace
 }  // namespace sasq
 
 extern "C" {
+
+int sasq_fakequant_fwd_bwd_static(const void* x, const void* grad_y, void* y, void* grad_x, float* grad_scale_dev,
+                                  int accumulate, int64_t numel, int dt, const float* scale_dev, int bits,
+                                  void* stream) {
+    using namespace sasq;
+    if (numel > kStaticMaxNumel) return SASQ_ERR_UNSUPPORTED;
+    if (numel < 0 || scale_dev == nullptr || grad_scale_dev == nullptr) return SASQ_ERR_INVALID_ARG;
+    if (bits < 2 || bits > 8 || (dt != SASQ_F16 && dt != SASQ_BF16)) return SASQ_ERR_INVALID_ARG;
+    if (numel > 0 && (x == nullptr || grad_y == nullptr || y == nullptr || grad_x == nullptr))
+        return SASQ_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(grad_y) || !aligned16(y) || !aligned16(grad_x)) return SASQ_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (numel == 0) {
+        if (!accumulate && cudaMemsetAsync(grad_scale_dev, 0, sizeof(float), st) != cudaSuccess) return SASQ_ERR_CUDA;
+        return SASQ_OK;
+    }
+    const int sm_count = device_sm_count_if_sm100();
+    if (sm_count <= 0) return SASQ_ERR_UNSUPPORTED;
+    const int grid = grid_for(numel, sm_count);
+    if (grid > kStaticPartials) return SASQ_ERR_UNSUPPORTED;      // more blocks than the static scratch holds
+    int err = SASQ_OK;
+    double* partials = static_partials_ptr(&err);                   // first call on a device resolves the address
+    if (partials == nullptr) return err;
+    int* status = status_word_ptr();
+    if (status == nullptr) return SASQ_ERR_CUDA;
+
+    QParams p{};
+    p.d[0].x = static_cast<const uint4*>(x);
+    p.d[0].g = static_cast<const uint4*>(grad_y);
+    p.d[0].y = static_cast<uint4*>(y);
+    p.d[0].dx = static_cast<uint4*>(grad_x);
+    p.d[0].numel = numel;
+    p.d[0].scale_index = 0;
+    p.n = 1;
+    p.scales = scale_dev;
+    p.partials = partials;      // every block overwrites its own slot: nothing has to start at zero
+    p.qn = (float)(1 << (bits - 1));
+    p.qp = (float)((1 << (bits - 1)) - 1);
+    p.status = status;
+    const cudaError_t e = (dt == SASQ_BF16) ? launch_mode<true>(true, true, p, grid, st)
+                                            : launch_mode<false>(true, true, p, grid, st);
+    if (e != cudaSuccess) return SASQ_ERR_CUDA;
+    CombineParams c{};
+    c.scale_index[0] = 0;
+    c.n = 1;
+    c.grid = grid;
+    c.accumulate_mask = accumulate ? 1u : 0u;
+    c.partials = partials;
+    c.grad_scales = grad_scale_dev;
+    fakequant_combine_kernel<<<1, kCombineThreads, 0, st>>>(c);
+    if (cudaGetLastError() != cudaSuccess) return SASQ_ERR_CUDA;
+    return SASQ_OK;
+}
 
 size_t sasq_fakequant_bwd_workspace(int64_t numel) {
     (void)numel;
