@@ -17,9 +17,15 @@ constexpr int kLoadHint = 1;
 constexpr int kStoreHint = 1;
 
 int* status_word_ptr() {
-    int* p = nullptr;
-    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_fakequant_status) != cudaSuccess) return nullptr;
-    return p;
+    static int* cache[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (cache[dev] == nullptr) {
+        int* p = nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_fakequant_status) != cudaSuccess) return nullptr;
+        cache[dev] = p;
+    }
+    return cache[dev];
 }
 
 template <bool BF, bool FWD, bool BWD>

@@ -9,6 +9,8 @@
 //   warps 2..5  epilogue: tcgen05.ld -> dequant -> 16-bit stores, overlapped with the next tile's mainloop
 // Every wait on an mbarrier is bounded; a wait that gives up raises SASQ_ERR_TIMEOUT
 // in the sticky status word and all roles fall through to the teardown.
+#include <mutex>
+
 #include "common.cuh"
 #include "tcgen05.cuh"
 
@@ -277,6 +279,363 @@ w8a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     }
 }
 
+
+// ---------------------------------------------------------------------------
+// CTA-pair kernel (cta_group::2): two CTAs on neighbouring SMs share one 256 x BN
+// output tile.  CTA r of the pair keeps rows [128 r, 128 r + 128) of A and rows
+// [BN/2 r, BN/2 (r+1)) of W in its own shared memory, so each byte of W is read
+// from shared memory by one SM only while feeding both tensor cores; at the int8
+// rate a single CTA's 128 x 256 tile needs more shared-memory bandwidth (TMA
+// writes + operand reads) than one SM has.  The leader CTA (rank 0) issues the
+// MMAs; completion is multicast to the barriers of both CTAs.
+// BN is chosen per problem (multiple of 16, at most 256) to fill whole waves.
+// ---------------------------------------------------------------------------
+constexpr int PBM = 256;                 // rows per pair tile
+#ifndef SASQ_PAIR_STAGES
+#define SASQ_PAIR_STAGES 5
+#endif
+constexpr int P_STAGES = SASQ_PAIR_STAGES;
+constexpr int P_A_BYTES = 128 * BK;      // per CTA: 128 rows of A
+constexpr int P_B_BYTES_MAX = 128 * BK;  // per CTA: up to 128 rows of W
+constexpr int P_STAGE_BYTES = P_A_BYTES + P_B_BYTES_MAX;
+
+constexpr int P_OUT_BUF_BYTES = 32 * 128;        // one epilogue warp's staging tile: 32 rows x 64 columns x 2 B
+constexpr int P_OUT_BYTES = 4 * 2 * P_OUT_BUF_BYTES;   // 4 warps, double buffered
+
+struct PairTail {
+    uint64_t full[P_STAGES];       // used in the leader: its producer arms it with the bytes of both CTAs' loads
+    uint64_t empty[P_STAGES];      // local: MMA of the pair has consumed the stage
+    uint64_t tmem_full[ACC_BUFS];  // local: accumulators of the tile are complete
+    uint64_t tmem_empty[ACC_BUFS]; // used in the leader: 8 epilogue warps (4 per CTA) have drained the buffer
+    float scale[256];
+    float bias[256];
+    uint32_t tmem_base;
+    volatile int abort_flag;
+};
+
+// the dynamic shared memory window of a CTA without static shared memory starts 1024-byte aligned; the kernel
+// checks this and reports SASQ_ERR_CUDA through the status word instead of running if it ever does not hold
+constexpr size_t kPairSmemBytes = (size_t)P_STAGES * P_STAGE_BYTES + P_OUT_BYTES + sizeof(PairTail);
+
+struct PairParams {
+    LinearParams lp;
+    int bn;             // tile width in output channels
+    int pair_m_blocks;  // ceil(T / 256)
+};
+
+__device__ __forceinline__ bool wait_bounded_pair(uint64_t* bar, uint32_t parity, PairTail* tail,
+                                                  const LinearParams& p) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    int polls = 0;
+    while (!ptx::mbar_try_wait(bar, parity)) {
+        if ((++polls & 63) == 0) {
+            if (tail->abort_flag) return false;
+            if (clock64() - t0 > p.wait_limit) {
+                tail->abort_flag = 1;
+                atomicMax(p.status, (int)SASQ_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+template <bool BF, int NCOLS>
+__device__ __forceinline__ void epilogue_chunk(const uint32_t* v, const float* scale, const float* bias, bool has_bias,
+                                               bool row_ok, int n_base, int N, uint16_t* yrow, int32_t* arow) {
+#pragma unroll
+    for (int j = 0; j < NCOLS; j += 8) {
+        if (row_ok && (n_base + j) < N) {
+            uint32_t o[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                float f0 = __fmul_rn(__int2float_rn((int)v[j + 2 * q]), scale[j + 2 * q]);
+                float f1 = __fmul_rn(__int2float_rn((int)v[j + 2 * q + 1]), scale[j + 2 * q + 1]);
+                if (has_bias) {
+                    f0 = __fadd_rn(f0, bias[j + 2 * q]);
+                    f1 = __fadd_rn(f1, bias[j + 2 * q + 1]);
+                }
+                o[q] = narrow2<BF>(f0, f1);
+            }
+            *reinterpret_cast<uint4*>(yrow + j) = make_uint4(o[0], o[1], o[2], o[3]);
+            if (arow != nullptr) {
+                *reinterpret_cast<uint4*>(arow + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                *reinterpret_cast<uint4*>(arow + j + 4) = make_uint4(v[j + 4], v[j + 5], v[j + 6], v[j + 7]);
+            }
+        }
+    }
+}
+
+template <bool BF>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
+                      const __grid_constant__ CUtensorMap tmap_y64, const __grid_constant__ CUtensorMap tmap_y16,
+                      const __grid_constant__ PairParams pp) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t* tiles = smem_raw;
+    uint8_t* out_stage = tiles + (size_t)P_STAGES * P_STAGE_BYTES;          // 1024-byte aligned
+    PairTail* tail = reinterpret_cast<PairTail*>(out_stage + P_OUT_BYTES);
+    const LinearParams& p = pp.lp;
+    if ((ptx::smem_u32(tiles) & 1023u) != 0) {      // uniform over the grid: every CTA returns before any barrier
+        if (threadIdx.x == 0) atomicMax(p.status, (int)SASQ_ERR_CUDA);
+        return;
+    }
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = ptx::cluster_ctarank();        // 0 = leader
+    const int bn = pp.bn;
+    const int half_bn = bn >> 1;
+    const uint32_t stage_tx = (uint32_t)(P_A_BYTES + half_bn * BK);   // bytes this CTA's two loads deliver
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < P_STAGES; ++s) {
+            ptx::mbar_init(&tail->full[s], 1);
+            ptx::mbar_init(&tail->empty[s], 1);
+        }
+        for (int b = 0; b < ACC_BUFS; ++b) {
+            ptx::mbar_init(&tail->tmem_full[b], 1);
+            ptx::mbar_init(&tail->tmem_empty[b], 8);
+        }
+        tail->abort_flag = 0;
+        ptx::mbar_init_fence();
+        ptx::prefetch_tensormap(&tmap_a);
+        ptx::prefetch_tensormap(&tmap_w);
+        ptx::prefetch_tensormap(&tmap_y64);
+        ptx::prefetch_tensormap(&tmap_y16);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc_pair(&tail->tmem_base, TMEM_COLS);
+        ptx::tmem_relinquish_pair();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::cluster_sync_all();            // both CTAs' barriers exist before anyone signals across the pair
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = tail->tmem_base;
+
+    const int n_blocks = (p.N + bn - 1) / bn;
+    const int num_tiles = pp.pair_m_blocks * n_blocks;
+    const int pair_id = blockIdx.x >> 1;
+    const int num_pairs = gridDim.x >> 1;
+
+    if (warp == 0) {
+        // ---------------- TMA producer (both CTAs) ----------------
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs) {
+            const int m_blk = tile % pp.pair_m_blocks, n_blk = tile / pp.pair_m_blocks;
+            const int a_row = m_blk * PBM + (int)rank * 128;
+            const int w_row = n_blk * bn + (int)rank * half_bn;
+            for (int kb = 0; kb < p.k_blocks && ok; ++kb) {
+                if (lane == 0) {
+                    ok = wait_bounded_pair(&tail->empty[stage], phase ^ 1u, tail, p);
+                    if (ok) {
+                        uint8_t* a_dst = tiles + (size_t)stage * P_STAGE_BYTES;
+                        uint8_t* b_dst = a_dst + P_A_BYTES;
+                        // Only the leader arms the barrier (with the bytes of both CTAs); the partner's copies
+                        // may complete first, which merely drives the transaction count negative for a while:
+                        // the phase cannot complete before the leader's arrival.
+                        const uint32_t full_leader = ptx::mapa_u32(ptx::smem_u32(&tail->full[stage]), 0);
+                        if (rank == 0) ptx::mbar_arrive_expect_tx(&tail->full[stage], 2u * stage_tx);
+                        ptx::tma_load_2d_pair(a_dst, &tmap_a, full_leader, kb * BK, a_row);
+                        ptx::tma_load_2d_pair(b_dst, &tmap_w, full_leader, kb * BK, w_row);
+                    }
+                }
+                ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
+                if (++stage == P_STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+        // after an abort, copies may still be in flight into this CTA's shared memory: their barrier lives in
+        // the leader, so give them a bounded grace period (a copy takes microseconds) before the CTA may exit
+        if (!ok) {
+            const long long t0 = clock64();
+            while (clock64() - t0 < (1LL << 22)) __nanosleep(1000);
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer (leader CTA only) ----------------
+        if (rank == 0) {
+            const uint32_t idesc = ptx::idesc_i8(PBM, bn);
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            int it = 0;
+            for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs, ++it) {
+                const int buf = it & 1;
+                const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+                if (lane == 0) ok = wait_bounded_pair(&tail->tmem_empty[buf], acc_phase ^ 1u, tail, p);
+                ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 256);
+                for (int kb = 0; kb < p.k_blocks && ok; ++kb) {
+                    if (lane == 0) {
+                        ok = wait_bounded_pair(&tail->full[stage], phase, tail, p);
+                        if (ok) {
+                            ptx::tc_fence_after_sync();
+                            const uint32_t a_addr = ptx::smem_u32(tiles + (size_t)stage * P_STAGE_BYTES);
+                            const uint64_t a_desc = ptx::smem_desc_k_major_sw128(a_addr);
+                            const uint64_t b_desc = ptx::smem_desc_k_major_sw128(a_addr + P_A_BYTES);
+#pragma unroll
+                            for (int k = 0; k < BK / UMMA_K; ++k) {
+                                ptx::mma_i8_ss_pair(d_tmem, a_desc + (uint64_t)(k * (UMMA_K >> 4)),
+                                                    b_desc + (uint64_t)(k * (UMMA_K >> 4)), idesc,
+                                                    (kb | k) != 0 ? 1u : 0u);
+                            }
+                            ptx::mma_commit_pair(&tail->empty[stage], 0x3);
+                            if (kb == p.k_blocks - 1) ptx::mma_commit_pair(&tail->tmem_full[buf], 0x3);
+                        }
+                    }
+                    ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
+                    if (++stage == P_STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else {
+        // ---------------- epilogue (warps 2..5 of both CTAs) ----------------
+        const int quad = warp & 3;
+        const int et = threadIdx.x - 64;
+        const float sx = __ldg(p.x_scale);
+        if (blockIdx.x == 0 && et == 0 && scale_is_bad(sx)) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
+        const bool has_bias = p.bias != nullptr;
+        bool ok = true;
+        int it = 0;
+        unsigned out_flip = 0;
+        for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs, ++it) {
+            const int m_blk = tile % pp.pair_m_blocks, n_blk = tile / pp.pair_m_blocks;
+            const int buf = it & 1;
+            const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+            const int n0 = n_blk * bn;
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            for (int j = et; j < bn; j += EPI_THREADS) {
+                const int n = n0 + j;
+                tail->scale[j] = (n < p.N) ? __fmul_rn(sx, __ldg(p.w_scale + n)) : 0.0f;
+                if (has_bias)
+                    tail->bias[j] = (n < p.N) ? widen1<BF>(__ldg(reinterpret_cast<const uint16_t*>(p.bias) + n)) : 0.0f;
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+
+            ok = wait_bounded_pair(&tail->tmem_full[buf], acc_phase, tail, p);
+            ok = epilogue_all_ok(ok);
+            if (!ok) break;
+            ptx::tc_fence_after_sync();
+
+            // Each warp owns 32 rows.  64 columns at a time: TMEM -> registers -> dequantise -> this warp's
+            // 128-byte-swizzled staging tile -> one TMA store (whole 128-byte lines; rows >= T and columns >= N
+            // are clipped by the tensor map).  A tile width that is not a multiple of 64 ends in 16-column pieces.
+            const int row0 = m_blk * PBM + (int)rank * 128 + quad * 32;
+            const int row = row0 + lane;
+            const bool row_ok = row < p.T;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * 256);
+            int32_t* arow = p.acc_out ? p.acc_out + (size_t)row * p.N + n0 : nullptr;
+            uint8_t* my_stage = out_stage + (size_t)quad * 2 * P_OUT_BUF_BYTES;
+            int c = 0;
+#pragma unroll 1
+            for (; c + 64 <= bn; c += 64) {
+                uint8_t* sbuf = my_stage + (size_t)(out_flip & 1) * P_OUT_BUF_BYTES;
+                if (lane == 0) ptx::bulk_wait_group_read<1>();      // the store that used this buffer has read it
+                __syncwarp();
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t v[32];
+                    ptx::tmem_ld_32x32(taddr + (uint32_t)(c + 32 * h), v);
+                    ptx::tmem_ld_wait();
+                    const float* sc = tail->scale + c + 32 * h;
+                    const float* bi = tail->bias + c + 32 * h;
+#pragma unroll
+                    for (int j = 0; j < 32; j += 8) {
+                        uint32_t o[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            float f0 = __fmul_rn(__int2float_rn((int)v[j + 2 * q]), sc[j + 2 * q]);
+                            float f1 = __fmul_rn(__int2float_rn((int)v[j + 2 * q + 1]), sc[j + 2 * q + 1]);
+                            if (has_bias) {
+                                f0 = __fadd_rn(f0, bi[j + 2 * q]);
+                                f1 = __fadd_rn(f1, bi[j + 2 * q + 1]);
+                            }
+                            o[q] = narrow2<BF>(f0, f1);
+                        }
+                        const int piece = 4 * h + (j >> 3);           // 16-byte piece of the 128-byte row
+                        *reinterpret_cast<uint4*>(sbuf + lane * 128 + ((piece ^ (lane & 7)) << 4)) =
+                            make_uint4(o[0], o[1], o[2], o[3]);
+                        if (arow != nullptr && row_ok && (n0 + c + 32 * h + j) < p.N) {
+                            int32_t* a = arow + c + 32 * h + j;
+                            *reinterpret_cast<uint4*>(a) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                            *reinterpret_cast<uint4*>(a + 4) = make_uint4(v[j + 4], v[j + 5], v[j + 6], v[j + 7]);
+                        }
+                    }
+                }
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    ptx::tma_store_2d(&tmap_y64, sbuf, n0 + c, row0);
+                    ptx::bulk_commit_group();
+                }
+                ++out_flip;
+            }
+#pragma unroll 1
+            for (; c < bn; c += 16) {       // 16-column pieces: 32-byte rows, 32-byte swizzle
+                uint8_t* sbuf = my_stage + (size_t)(out_flip & 1) * P_OUT_BUF_BYTES;
+                if (lane == 0) ptx::bulk_wait_group_read<1>();
+                __syncwarp();
+                uint32_t v[16];
+                ptx::tmem_ld_32x16(taddr + (uint32_t)c, v);
+                ptx::tmem_ld_wait();
+                const float* sc = tail->scale + c;
+                const float* bi = tail->bias + c;
+#pragma unroll
+                for (int j = 0; j < 16; j += 8) {
+                    uint32_t o[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        float f0 = __fmul_rn(__int2float_rn((int)v[j + 2 * q]), sc[j + 2 * q]);
+                        float f1 = __fmul_rn(__int2float_rn((int)v[j + 2 * q + 1]), sc[j + 2 * q + 1]);
+                        if (has_bias) {
+                            f0 = __fadd_rn(f0, bi[j + 2 * q]);
+                            f1 = __fadd_rn(f1, bi[j + 2 * q + 1]);
+                        }
+                        o[q] = narrow2<BF>(f0, f1);
+                    }
+                    const int piece = j >> 3;
+                    *reinterpret_cast<uint4*>(sbuf + lane * 32 + ((piece ^ ((lane >> 2) & 1)) << 4)) =
+                        make_uint4(o[0], o[1], o[2], o[3]);
+                    if (arow != nullptr && row_ok && (n0 + c + j) < p.N) {
+                        int32_t* a = arow + c + j;
+                        *reinterpret_cast<uint4*>(a) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                        *reinterpret_cast<uint4*>(a + 4) = make_uint4(v[j + 4], v[j + 5], v[j + 6], v[j + 7]);
+                    }
+                }
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    ptx::tma_store_2d(&tmap_y16, sbuf, n0 + c, row0);
+                    ptx::bulk_commit_group();
+                }
+                ++out_flip;
+            }
+            // this warp has drained the accumulator buffer: tell the leader's MMA issuer
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(ptx::mapa_u32(ptx::smem_u32(&tail->tmem_empty[buf]), 0));
+        }
+        if (lane == 0) ptx::bulk_wait_group_all();      // output stores have left shared memory and are performed
+    }
+
+    // ---------------- teardown ----------------
+    // Neither CTA may leave while its partner can still read its shared memory, signal its barriers or
+    // run MMAs into its TMEM.  The epilogues of both CTAs have seen the last tile's accumulators complete
+    // (or every role has given up after a bounded wait), so a pair-wide barrier is enough.
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::cluster_sync_all();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc_pair(tmem_base, TMEM_COLS);
+    }
+}
+
 // Eq. 1 with the fixed factor, written once to int8 (operand A of the GEMM).
 // 16 elements per thread: two 128-bit loads, one 128-bit store.
 template <bool BF>
@@ -321,23 +680,136 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// int8 [rows, K] row-major -> tiles of box_rows x 128 bytes, 128-byte swizzle, zero fill outside
-bool make_tmap(CUtensorMap* m, const void* base, long long rows, long long K, int box_rows) {
+// int8 [rows, K] row-major -> tiles of box_rows x 128 bytes, 128-byte swizzle, zero fill outside.
+// Encoding a map costs a few microseconds on the host, which matters for decode-sized calls; weights are
+// frozen and workspaces are reused, so the last few maps are kept (keyed by everything that defines them).
+struct TmapKey {
+    const void* base;
+    long long rows, cols;
+    int box_rows, box_cols, elem_bytes;
+};
+struct TmapEntry {
+    TmapKey key;
+    CUtensorMap map;
+    bool valid;
+};
+constexpr int kTmapCache = 64;
+std::mutex g_tmap_mutex;
+TmapEntry g_tmap_cache[kTmapCache];
+int g_tmap_next = 0;
+
+// [rows, cols] row-major tensor of 1- or 2-byte elements, box of box_rows x box_cols whose inner extent is
+// 32, 64 or 128 bytes and selects the matching swizzle
+bool make_tmap_generic(CUtensorMap* m, const void* base, long long rows, long long cols, int box_rows, int box_cols,
+                       int elem_bytes) {
+    {
+        std::lock_guard<std::mutex> lock(g_tmap_mutex);
+        for (int i = 0; i < kTmapCache; ++i) {
+            const TmapEntry& e = g_tmap_cache[i];
+            if (e.valid && e.key.base == base && e.key.rows == rows && e.key.cols == cols &&
+                e.key.box_rows == box_rows && e.key.box_cols == box_cols && e.key.elem_bytes == elem_bytes) {
+                *m = e.map;
+                return true;
+            }
+        }
+    }
     EncodeTiledFn fn = encode_fn();
     if (fn == nullptr) return false;
-    cuuint64_t gdim[2] = {(cuuint64_t)K, (cuuint64_t)rows};
-    cuuint64_t gstride[1] = {(cuuint64_t)K};
-    cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+    const int inner = box_cols * elem_bytes;
+    const CUtensorMapSwizzle sw = inner == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                : inner == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                              : CU_TENSOR_MAP_SWIZZLE_32B;
+    cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t gstride[1] = {(cuuint64_t)(cols * elem_bytes)};
+    cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), gdim, gstride, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    if (fn(m, elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_UINT16, 2,
+           const_cast<void*>(base), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    std::lock_guard<std::mutex> lock(g_tmap_mutex);
+    TmapEntry& e = g_tmap_cache[g_tmap_next];
+    g_tmap_next = (g_tmap_next + 1) % kTmapCache;
+    e.key = TmapKey{base, rows, cols, box_rows, box_cols, elem_bytes};
+    e.map = *m;
+    e.valid = true;
+    return true;
+}
+
+// int8 operand [rows, K]: boxes of box_rows x 128 bytes
+bool make_tmap(CUtensorMap* m, const void* base, long long rows, long long K, int box_rows) {
+    return make_tmap_generic(m, base, rows, K, box_rows, BK, 1);
+}
+// 16-bit output [T, N]: boxes of 32 rows x box_cols columns (one epilogue warp's rows)
+bool make_tmap_out(CUtensorMap* m, const void* base, long long T, long long N, int box_cols) {
+    return make_tmap_generic(m, base, T, N, 32, box_cols, 2);
+}
+
+// Number of CTA pairs that can be resident at once (one pair per TPC); also opts the kernel in to its shared memory.
+int pair_capacity(bool bf, int sm_count) {
+    static int cache[64][2] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
+    if (cache[dev][bf] != 0) return cache[dev][bf];
+    const void* fn = bf ? reinterpret_cast<const void*>(w8a8_gemm_pair_kernel<true>)
+                        : reinterpret_cast<const void*>(w8a8_gemm_pair_kernel<false>);
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemBytes) != cudaSuccess)
+        return -1;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)sm_count, 1, 1);
+    cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = kPairSmemBytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&clusters, fn, &cfg) != cudaSuccess || clusters <= 0) clusters = sm_count / 2;
+    if (clusters > sm_count / 2) clusters = sm_count / 2;
+    cache[dev][bf] = clusters;
+    return clusters;
+}
+
+// Tile width (multiple of 16, 128..256) that minimises waves x width for this problem on `pairs` CTA pairs.
+int choose_bn(int pair_m_blocks, int N, int pairs) {
+    int best = 256;
+    long long best_cost = -1;
+    for (int bn = 256; bn >= 128; bn -= 16) {
+        const long long tiles = (long long)pair_m_blocks * ((N + bn - 1) / bn);
+        const long long waves = (tiles + pairs - 1) / pairs;
+        const long long cost = waves * bn;
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = bn; }
+    }
+    return best;
 }
 
 int* status_word_ptr() {
-    int* p = nullptr;
-    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_linear_status) != cudaSuccess) return nullptr;
-    return p;
+    static int* cache[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (cache[dev] == nullptr) {
+        int* p = nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_linear_status) != cudaSuccess) return nullptr;
+        cache[dev] = p;
+    }
+    return cache[dev];
+}
+
+// opts the single-CTA kernel in to its shared memory once per device
+bool single_kernel_ready(bool bf) {
+    static bool done[64][2] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    if (done[dev][bf]) return true;
+    const void* fn = bf ? reinterpret_cast<const void*>(w8a8_gemm_kernel<true>)
+                        : reinterpret_cast<const void*>(w8a8_gemm_kernel<false>);
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess)
+        return false;
+    done[dev][bf] = true;
+    return true;
 }
 
 }  // namespace
@@ -393,8 +865,6 @@ int sasq_static_w8a8_linear(const void* x, const int8_t* w, const float* w_scale
     }
 
     // 2. TMA-fed tcgen05 GEMM with the dequant epilogue
-    CUtensorMap tmap_a, tmap_w;
-    if (!make_tmap(&tmap_a, a_int8, T, K, BM) || !make_tmap(&tmap_w, w, N, K, BN)) return SASQ_ERR_CUDA;
     LinearParams p{};
     p.w_scale = w_scale;
     p.x_scale = x_scale_dev;
@@ -402,22 +872,50 @@ int sasq_static_w8a8_linear(const void* x, const int8_t* w, const float* w_scale
     p.y = y;
     p.acc_out = acc_out;
     p.T = (int)T; p.N = (int)N; p.K = (int)K;
-    p.m_blocks = (int)((T + BM - 1) / BM);
-    p.n_blocks = (int)((N + BN - 1) / BN);
     p.k_blocks = (int)((K + BK - 1) / BK);
     p.status = status;
     p.wait_limit = kWaitLimit;
-    const long long tiles = (long long)p.m_blocks * p.n_blocks;
-    const int grid = (int)(tiles < sm_count ? tiles : sm_count);
+    CUtensorMap tmap_a, tmap_w;
     cudaError_t e;
-    if (dt == SASQ_BF16) {
-        e = cudaFuncSetAttribute(w8a8_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (T > BM) {
+        // CTA pairs, 256 x bn tiles; bn minimises (waves x bn) over the resident pairs
+        const int pairs = pair_capacity(dt == SASQ_BF16, sm_count);
+        if (pairs <= 0) return SASQ_ERR_CUDA;
+        PairParams pp{};
+        pp.pair_m_blocks = (int)((T + PBM - 1) / PBM);
+        pp.bn = choose_bn(pp.pair_m_blocks, (int)N, pairs);
+        p.m_blocks = pp.pair_m_blocks;
+        p.n_blocks = (int)((N + pp.bn - 1) / pp.bn);
+        pp.lp = p;
+        if (!make_tmap(&tmap_a, a_int8, T, K, 128) || !make_tmap(&tmap_w, w, N, K, pp.bn / 2)) return SASQ_ERR_CUDA;
+        CUtensorMap tmap_y64, tmap_y16;
+        if (!make_tmap_out(&tmap_y64, y, T, N, 64) || !make_tmap_out(&tmap_y16, y, T, N, 16)) return SASQ_ERR_CUDA;
+        const long long tiles = (long long)p.m_blocks * p.n_blocks;
+        const int grid = 2 * (int)(tiles < pairs ? tiles : pairs);
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((unsigned)grid, 1, 1);
+        cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+        cfg.dynamicSmemBytes = kPairSmemBytes;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (dt == SASQ_BF16) e = cudaLaunchKernelEx(&cfg, w8a8_gemm_pair_kernel<true>, tmap_a, tmap_w, tmap_y64, tmap_y16, pp);
+        else e = cudaLaunchKernelEx(&cfg, w8a8_gemm_pair_kernel<false>, tmap_a, tmap_w, tmap_y64, tmap_y16, pp);
         if (e != cudaSuccess) return SASQ_ERR_CUDA;
-        w8a8_gemm_kernel<true><<<grid, NUM_THREADS, kSmemBytes, st>>>(tmap_a, tmap_w, p);
     } else {
-        e = cudaFuncSetAttribute(w8a8_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-        if (e != cudaSuccess) return SASQ_ERR_CUDA;
-        w8a8_gemm_kernel<false><<<grid, NUM_THREADS, kSmemBytes, st>>>(tmap_a, tmap_w, p);
+        p.m_blocks = (int)((T + BM - 1) / BM);
+        p.n_blocks = (int)((N + BN - 1) / BN);
+        if (!make_tmap(&tmap_a, a_int8, T, K, BM) || !make_tmap(&tmap_w, w, N, K, BN)) return SASQ_ERR_CUDA;
+        const long long tiles = (long long)p.m_blocks * p.n_blocks;
+        const int grid = (int)(tiles < sm_count ? tiles : sm_count);
+        if (!single_kernel_ready(dt == SASQ_BF16)) return SASQ_ERR_CUDA;
+        if (dt == SASQ_BF16) w8a8_gemm_kernel<true><<<grid, NUM_THREADS, kSmemBytes, st>>>(tmap_a, tmap_w, p);
+        else w8a8_gemm_kernel<false><<<grid, NUM_THREADS, kSmemBytes, st>>>(tmap_a, tmap_w, p);
     }
     if (cudaGetLastError() != cudaSuccess) return SASQ_ERR_CUDA;
     return SASQ_OK;
