@@ -18,7 +18,7 @@ __all__ = [
     "sasq_fakequant_fwd", "sasq_fakequant_bwd_workspace", "sasq_fakequant_bwd", "sasq_fakequant_fwd_bwd",
     "sasq_fakequant_multi_workspace", "sasq_fakequant_fwd_bwd_multi", "sasq_static_w8a8_linear_workspace",
     "sasq_static_w8a8_linear", "sasq_device_status", "QDesc", "sasq_absmax_scale_workspace", "sasq_absmax_scale",
-    "sasq_quantize_weight", "LAUNCHES_PER_LINEAR", "sasq_fakequant_fwd_bwd_static",
+    "sasq_quantize_weight", "LAUNCHES_PER_LINEAR", "sasq_fakequant_fwd_bwd_static", "sasq_static_w8a8_linear_tiles",
 ]
 
 SASQ_F16 = 0
@@ -78,6 +78,8 @@ def load_library() -> ctypes.CDLL:
     L.sasq_static_w8a8_linear_workspace.argtypes = [i64, i64, i64]
     L.sasq_static_w8a8_linear.restype = i32
     L.sasq_static_w8a8_linear.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, sz, vp]
+    L.sasq_static_w8a8_linear_tiles.restype = i32
+    L.sasq_static_w8a8_linear_tiles.argtypes = [i64, i64, i32, i32, ctypes.POINTER(ctypes.c_int32), i32]
     L.sasq_device_status.restype = i32
     L.sasq_device_status.argtypes = [vp]
     L.sasq_absmax_scale_workspace.restype = sz
@@ -232,6 +234,17 @@ def sasq_static_w8a8_linear(x, w, w_scale, x_scale, y, bias=None, acc_out=None, 
     _check(load_library().sasq_static_w8a8_linear(_ptr(x), _ptr(w), _ptr(w_scale), _ptr(x_scale), _ptr(bias), _ptr(y),
                                                   _ptr(acc_out), T, N, K, _dt(x), int(bits), _ptr(workspace),
                                                   _nbytes(workspace), _stream(stream)), "sasq_static_w8a8_linear")
+
+
+def sasq_static_w8a8_linear_tiles(T: int, N: int, num_pairs: int, pair_id: int):
+    """Tiles (first row, first column, width) that CTA pair `pair_id` of `num_pairs` walks for a [T, N] output."""
+    L = load_library()
+    n = L.sasq_static_w8a8_linear_tiles(int(T), int(N), int(num_pairs), int(pair_id), None, 0)
+    if n < 0:
+        raise ValueError("invalid arguments")
+    buf = (ctypes.c_int32 * (3 * max(n, 1)))()
+    L.sasq_static_w8a8_linear_tiles(int(T), int(N), int(num_pairs), int(pair_id), buf, n)
+    return [(buf[3 * i], buf[3 * i + 1], buf[3 * i + 2]) for i in range(n)]
 
 
 def sasq_device_status(stream=None) -> int:

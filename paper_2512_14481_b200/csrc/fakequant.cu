@@ -1,4 +1,6 @@
 // C-ABI entry points of the fake-quant forward / backward / fused path.
+#include <atomic>
+
 #include "fakequant_kernels.cuh"
 
 namespace sasq {
@@ -26,6 +28,25 @@ int* status_word_ptr() {
         cache[dev] = p;
     }
     return cache[dev];
+}
+
+// Ticket counters of the second reduction stage.  They are zero when the library is loaded and every launch
+// leaves the one it used at zero again.  Launches draw them round-robin, so two launches share a counter only if
+// more than kTicketSlots launches of this library were executing at the same time, which no GPU does.
+constexpr unsigned kTicketSlots = 256;
+static __device__ unsigned g_tickets[kTicketSlots];
+
+unsigned* next_ticket() {
+    static unsigned* base[64] = {nullptr};
+    static std::atomic<unsigned> next{0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (base[dev] == nullptr) {
+        unsigned* p = nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_tickets) != cudaSuccess) return nullptr;
+        base[dev] = p;
+    }
+    return base[dev] + (next.fetch_add(1u, std::memory_order_relaxed) % kTicketSlots);
 }
 
 template <bool BF, bool FWD, bool BWD>
@@ -92,7 +113,6 @@ int run_multi(const sasq_qdesc_t* descs, int n_tensors, const float* scales_dev,
     for (int base = 0; base < n_tensors; base += kMaxDescsPerLaunch) {
         const int n = (n_tensors - base < kMaxDescsPerLaunch) ? (n_tensors - base) : kMaxDescsPerLaunch;
         QParams p{};
-        CombineParams c{};
         for (int i = 0; i < n; ++i) {
             const sasq_qdesc_t& d = descs[base + i];
             p.d[i].x = static_cast<const uint4*>(d.x);
@@ -101,10 +121,9 @@ int run_multi(const sasq_qdesc_t* descs, int n_tensors, const float* scales_dev,
             p.d[i].dx = static_cast<uint4*>(d.grad_x);
             p.d[i].numel = d.numel;
             p.d[i].scale_index = d.scale_index;
-            c.scale_index[i] = d.scale_index;
             bool seen_before = false;
             for (int k = 0; k < base && !seen_before; ++k) seen_before = (descs[k].scale_index == d.scale_index);
-            if (accumulate || seen_before) c.accumulate_mask |= (1u << i);
+            if (accumulate || seen_before) p.accumulate_mask |= (1u << i);
         }
         p.n = n;
         p.scales = scales_dev;
@@ -112,17 +131,14 @@ int run_multi(const sasq_qdesc_t* descs, int n_tensors, const float* scales_dev,
         p.qn = (float)(1 << (bits - 1));
         p.qp = (float)((1 << (bits - 1)) - 1);
         p.status = status;
+        p.grad_scales = grad_scales_dev;
+        if (bwd) {
+            p.ticket = next_ticket();
+            if (p.ticket == nullptr) return SASQ_ERR_CUDA;
+        }
         cudaError_t e = (dt == SASQ_BF16) ? launch_mode<true>(fwd, bwd, p, grid, st)
                                           : launch_mode<false>(fwd, bwd, p, grid, st);
         if (e != cudaSuccess) return SASQ_ERR_CUDA;
-        if (bwd) {
-            c.n = n;
-            c.grid = grid;
-            c.partials = p.partials;
-            c.grad_scales = grad_scales_dev;
-            fakequant_combine_kernel<<<n, kCombineThreads, 0, st>>>(c);
-            if (cudaGetLastError() != cudaSuccess) return SASQ_ERR_CUDA;
-        }
     }
     return SASQ_OK;
 }
@@ -226,18 +242,13 @@ int sasq_fakequant_fwd_bwd_static(const void* x, const void* grad_y, void* y, vo
     p.qn = (float)(1 << (bits - 1));
     p.qp = (float)((1 << (bits - 1)) - 1);
     p.status = status;
+    p.grad_scales = grad_scale_dev;
+    p.accumulate_mask = accumulate ? 1u : 0u;
+    p.ticket = next_ticket();
+    if (p.ticket == nullptr) return SASQ_ERR_CUDA;
     const cudaError_t e = (dt == SASQ_BF16) ? launch_mode<true>(true, true, p, grid, st)
                                             : launch_mode<false>(true, true, p, grid, st);
     if (e != cudaSuccess) return SASQ_ERR_CUDA;
-    CombineParams c{};
-    c.scale_index[0] = 0;
-    c.n = 1;
-    c.grid = grid;
-    c.accumulate_mask = accumulate ? 1u : 0u;
-    c.partials = partials;
-    c.grad_scales = grad_scale_dev;
-    fakequant_combine_kernel<<<1, kCombineThreads, 0, st>>>(c);
-    if (cudaGetLastError() != cudaSuccess) return SASQ_ERR_CUDA;
     return SASQ_OK;
 }
 

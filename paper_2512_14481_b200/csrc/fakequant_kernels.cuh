@@ -9,7 +9,8 @@
 // 128-bit stores of y and dx, and a deterministic reduction of ds:
 // fp32 tree over the 8 products of a vector -> double per thread -> warp
 // shuffles -> shared memory -> one double per (tensor, block) in the workspace.
-// A second tiny kernel adds the block partials in a fixed order.
+// The block that finishes last (a ticket counter) adds the block partials in a
+// fixed order and writes the gradients: one launch, no second pass.
 //
 // The path is HBM-bound: 4 B / element forward, 6 B backward, 8 B fused.
 #pragma once
@@ -39,6 +40,10 @@ struct QParams {
     float qn;                // 2^(b-1)
     float qp;                // 2^(b-1) - 1
     int* status;
+    // second stage (backward only)
+    float* grad_scales;
+    unsigned* ticket;        // zero before the launch; the last block leaves it zero again
+    unsigned accumulate_mask; // bit j: descriptor j's slot is added to, not overwritten
 };
 
 struct Quant2 {
@@ -183,39 +188,56 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) fakequant_kernel(const __
             if (threadIdx.x == 0) p.partials[(long long)ti * gridDim.x + blockIdx.x] = tot;
         }
     }
-}
 
-// Second stage: block j acts iff descriptor j is the first of its factor slot in
-// this launch; it adds the partials of every descriptor of that slot, in
-// descriptor order then block order, and writes (or adds to) grad_scales[slot].
-struct CombineParams {
-    int scale_index[kMaxDescsPerLaunch];
-    int n;
-    int grid;                 // partials per descriptor
-    unsigned accumulate_mask; // bit j: descriptor j's slot is added to, not overwritten
-    const double* partials;
-    float* grad_scales;
-};
-
-constexpr int kCombineThreads = 256;
-
-__global__ void __launch_bounds__(kCombineThreads) fakequant_combine_kernel(const __grid_constant__ CombineParams p) {
-    __shared__ double warp_sums[kCombineThreads / 32];
-    const int j = blockIdx.x;
-    const int slot = p.scale_index[j];
-    if (slot < 0) return;                                   // descriptor without a backward part
-    for (int k = 0; k < j; ++k)
-        if (p.scale_index[k] == slot) return;               // not the first of its slot
-    double acc = 0.0;
-    for (int k = j; k < p.n; ++k) {
-        if (p.scale_index[k] != slot) continue;
-        const double* part = p.partials + (long long)k * p.grid;
-        for (int i = threadIdx.x; i < p.grid; i += kCombineThreads) acc += part[i];
-    }
-    const double tot = block_sum_fixed<kCombineThreads>(acc, warp_sums);
-    if (threadIdx.x == 0) {
-        const float prev = ((p.accumulate_mask >> j) & 1u) ? p.grad_scales[slot] : 0.0f;
-        p.grad_scales[slot] = prev + (float)tot;
+    if constexpr (BWD) {
+        // Second stage, by whichever block finishes last.  Warp w totals the partials of descriptors w, w + W, ...:
+        // per lane blocks lane, lane + 32, ... in that order (loads issued 16 at a time so that their latencies
+        // overlap), then the xor-shuffle tree.  Then one lane per factor slot adds the totals of the descriptors
+        // that share the slot, in descriptor order.  The order depends only on the launch shape, so the result
+        // is bit-identical from run to run.
+        __shared__ unsigned s_ticket;
+        __shared__ double s_total[kMaxDescsPerLaunch];
+        if (threadIdx.x == 0) {
+            __threadfence();                                   // this block's partials before its ticket
+            s_ticket = atomicAdd(p.ticket, 1u);
+        }
+        __syncthreads();
+        if (s_ticket != gridDim.x - 1) return;
+        __threadfence();                                       // every other block's partials after their tickets
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        const int nblk = (int)gridDim.x;
+        for (int j = warp; j < p.n; j += THREADS / 32) {
+            const double* part = p.partials + (long long)j * nblk;
+            double acc = 0.0;
+            for (int i0 = lane; i0 < nblk; i0 += 32 * 16) {
+                double v[16];
+#pragma unroll
+                for (int u = 0; u < 16; ++u) {
+                    const int i = i0 + 32 * u;
+                    v[u] = (i < nblk) ? __ldcg(part + i) : 0.0;
+                }
+#pragma unroll
+                for (int u = 0; u < 16; ++u) acc += v[u];
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
+            if (lane == 0) s_total[j] = acc;
+        }
+        __syncthreads();
+        if (threadIdx.x < p.n) {
+            const int j = threadIdx.x;
+            const int slot = p.d[j].scale_index;
+            bool first = true;
+            for (int k = 0; k < j; ++k) first = first && (p.d[k].scale_index != slot);
+            if (first) {
+                double tot = 0.0;
+                for (int k = j; k < p.n; ++k)
+                    if (p.d[k].scale_index == slot) tot += s_total[k];
+                const float prev = ((p.accumulate_mask >> j) & 1u) ? p.grad_scales[slot] : 0.0f;
+                p.grad_scales[slot] = prev + (float)tot;
+            }
+        }
+        if (threadIdx.x == 0) *p.ticket = 0u;                  // ready for the next launch that draws this counter
     }
 }
 

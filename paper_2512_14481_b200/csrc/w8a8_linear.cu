@@ -3,10 +3,13 @@
 //   acc   = X_int * W_int^T                      int8 x int8 -> int32 on tcgen05 tensor cores, accumulators in TMEM
 //   y     = narrow(fl32(acc) * fl32(s_x * s_w[n]) (+ bias[n]))
 //
-// Persistent, warp-specialised kernel, one CTA per SM:
-//   warp 0      TMA producer: W tiles (and pre-quantized A tiles) -> 128-byte-swizzled shared memory
-//   warp 1      MMA issuer: tcgen05.mma.kind::i8, 128 x 256 x 32 per instruction, TMEM double-buffered
+// Persistent, warp-specialised kernels, one CTA per SM:
+//   warp 0      TMA producer: W tiles and int8 A tiles -> 128-byte-swizzled shared memory
+//   warp 1      MMA issuer: tcgen05.mma.kind::i8, 32 bytes of K per instruction, TMEM double-buffered
 //   warps 2..5  epilogue: tcgen05.ld -> dequant -> 16-bit stores, overlapped with the next tile's mainloop
+//   warps 6..9  (CTA-pair kernel) activation quantizer: Eq. 1 with the fixed factor on rows of x -> int8 A in the
+//               workspace, published per 256-row block; the producers wait for the block they are about to load,
+//               so the quantization of later rows runs under the MMAs of earlier ones and costs no launch
 // Every wait on an mbarrier is bounded; a wait that gives up raises SASQ_ERR_TIMEOUT
 // in the sticky status word and all roles fall through to the teardown.
 #include <mutex>
@@ -25,6 +28,7 @@ constexpr int BM = 128;            // rows of x per tile (UMMA M)
 constexpr int BN = 256;            // output channels per tile (UMMA N)
 constexpr int BK = 128;            // int8 elements (= bytes) of K per pipeline stage: one 128-byte swizzle row
 constexpr int UMMA_K = 32;         // K per tcgen05.mma.kind::i8
+static_assert(BK / UMMA_K == 4, "the issue loops are written for four MMAs per stage");
 constexpr int STAGES = 4;
 constexpr int ACC_BUFS = 2;        // TMEM accumulator buffers (2 x 256 columns = all 512)
 constexpr int A_STAGE_BYTES = BM * BK;
@@ -133,76 +137,73 @@ w8a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
-        int stage = 0;
-        uint32_t phase = 0;
-        bool ok = true;
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-            const int m_blk = tile % p.m_blocks, n_blk = tile / p.m_blocks;
-            for (int kb = 0; kb < p.k_blocks && ok; ++kb) {
-                if (lane == 0) {
+        if (ptx::elect_one()) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                const int m_blk = tile % p.m_blocks, n_blk = tile / p.m_blocks;
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
                     ok = wait_bounded(&tail->empty[stage], phase ^ 1u, tail, p);
-                    if (ok) {
-                        uint8_t* a_dst = tiles + (size_t)stage * STAGE_BYTES;
-                        uint8_t* b_dst = a_dst + A_STAGE_BYTES;
-                        ptx::mbar_arrive_expect_tx(&tail->full[stage], STAGE_BYTES);
-                        ptx::tma_load_2d(a_dst, &tmap_a, &tail->full[stage], kb * BK, m_blk * BM);
-                        ptx::tma_load_2d(b_dst, &tmap_w, &tail->full[stage], kb * BK, n_blk * BN);
+                    if (!ok) break;
+                    uint8_t* a_dst = tiles + (size_t)stage * STAGE_BYTES;
+                    uint8_t* b_dst = a_dst + A_STAGE_BYTES;
+                    ptx::mbar_arrive_expect_tx(&tail->full[stage], STAGE_BYTES);
+                    ptx::tma_load_2d(a_dst, &tmap_a, &tail->full[stage], kb * BK, m_blk * BM);
+                    ptx::tma_load_2d(b_dst, &tmap_w, &tail->full[stage], kb * BK, n_blk * BN);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+            // teardown: copies still in flight must land before the CTA's shared memory goes away.
+            // Every armed full barrier either was consumed already (wait returns at once) or completes here.
+            if (!ok) {
+                for (int s = 0; s < STAGES; ++s) {
+                    const long long t0 = clock64();
+                    // the phase armed last for stage s: stages before `stage` are in `phase`, the others in phase^1
+                    const uint32_t par = (s < stage) ? phase : (phase ^ 1u);
+                    while (!ptx::mbar_try_wait(&tail->full[s], par)) {
+                        if (clock64() - t0 > (1LL << 24)) break;
                     }
                 }
-                ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
         }
-        // teardown: copies still in flight must land before the CTA's shared memory goes away.
-        // Every armed full barrier either was consumed already (wait returns at once) or completes here.
-        if (lane == 0 && !ok) {
-            for (int s = 0; s < STAGES; ++s) {
-                const long long t0 = clock64();
-                // the phase armed last for stage s: stages before `stage` are in `phase`, the others in phase^1
-                const uint32_t par = (s < stage) ? phase : (phase ^ 1u);
-                while (!ptx::mbar_try_wait(&tail->full[s], par)) {
-                    if (clock64() - t0 > (1LL << 24)) break;
-                }
-            }
-        }
+        __syncwarp();
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        constexpr uint32_t idesc = ptx::idesc_i8(BM, BN);
-        int stage = 0;
-        uint32_t phase = 0;
-        bool ok = true;
-        int it = 0;
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
-            const int buf = it & 1;
-            const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-            if (lane == 0) ok = wait_bounded(&tail->tmem_empty[buf], acc_phase ^ 1u, tail, p);
-            ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
-            if (!ok) break;
-            ptx::tc_fence_after_sync();
-            const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
-            for (int kb = 0; kb < p.k_blocks && ok; ++kb) {
-                if (lane == 0) {
+        if (ptx::elect_one()) {
+            constexpr uint32_t idesc = ptx::idesc_i8(BM, BN);
+            const uint64_t a_desc0 = ptx::smem_desc_k_major_sw128(ptx::smem_u32(tiles));
+            const uint64_t b_desc0 = ptx::smem_desc_k_major_sw128(ptx::smem_u32(tiles) + A_STAGE_BYTES);
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            int it = 0;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+                const int buf = it & 1;
+                const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+                ok = wait_bounded(&tail->tmem_empty[buf], acc_phase ^ 1u, tail, p);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+                uint32_t accumulate = 0;
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
                     ok = wait_bounded(&tail->full[stage], phase, tail, p);
-                    if (ok) {
-                        ptx::tc_fence_after_sync();
-                        const uint32_t a_addr = ptx::smem_u32(tiles + (size_t)stage * STAGE_BYTES);
-                        const uint32_t b_addr = a_addr + A_STAGE_BYTES;
-                        const uint64_t a_desc = ptx::smem_desc_k_major_sw128(a_addr);
-                        const uint64_t b_desc = ptx::smem_desc_k_major_sw128(b_addr);
-#pragma unroll
-                        for (int k = 0; k < BK / UMMA_K; ++k) {
-                            // advance both operands by 32 bytes of K inside the swizzled row
-                            ptx::mma_i8_ss(d_tmem, a_desc + (uint64_t)(k * (UMMA_K >> 4)),
-                                           b_desc + (uint64_t)(k * (UMMA_K >> 4)), idesc, (kb | k) != 0 ? 1u : 0u);
-                        }
-                        ptx::mma_commit(&tail->empty[stage]);          // stage reusable once these MMAs are done
-                        if (kb == p.k_blocks - 1) ptx::mma_commit(&tail->tmem_full[buf]);
-                    }
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
+                    const uint64_t a_desc = a_desc0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
+                    const uint64_t b_desc = b_desc0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
+                    ptx::mma_i8_ss(d_tmem, a_desc, b_desc, idesc, accumulate);
+                    ptx::mma_i8_ss_acc(d_tmem, a_desc + 2, b_desc + 2, idesc);
+                    ptx::mma_i8_ss_acc(d_tmem, a_desc + 4, b_desc + 4, idesc);
+                    ptx::mma_i8_ss_acc(d_tmem, a_desc + 6, b_desc + 6, idesc);
+                    accumulate = 1u;
+                    ptx::mma_commit(&tail->empty[stage]);          // stage reusable once these MMAs are done
+                    if (kb == p.k_blocks - 1) ptx::mma_commit(&tail->tmem_full[buf]);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
-                ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
         }
+        __syncwarp();
     } else {
         // ---------------- epilogue (warps 2..5) ----------------
         const int quad = warp & 3;                      // TMEM lane quadrant this warp may read
@@ -288,7 +289,16 @@ w8a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 // rate a single CTA's 128 x 256 tile needs more shared-memory bandwidth (TMA
 // writes + operand reads) than one SM has.  The leader CTA (rank 0) issues the
 // MMAs; completion is multicast to the barriers of both CTAs.
-// BN is chosen per problem (multiple of 16, at most 256) to fill whole waves.
+//
+// Tiling: every 256-row block of the output is cut into the same number of
+// column tiles whose widths are multiples of 16 and differ by at most 16, so
+// no tile is ragged; that number is chosen per problem so that the tiles fill
+// whole waves of the resident pairs (plan_pair_tiles).
+//
+// The tensor pipe takes the next MMA only when the one before it is nearly
+// done, so whatever the issuing lane does between two MMAs is time the pipe
+// idles: the issue loop runs in one elected lane with nothing in it but the
+// barrier poll, two descriptor adds, the MMAs and the commit.
 // ---------------------------------------------------------------------------
 constexpr int PBM = 256;                 // rows per pair tile
 #ifndef SASQ_PAIR_STAGES
@@ -298,6 +308,12 @@ constexpr int P_STAGES = SASQ_PAIR_STAGES;
 constexpr int P_A_BYTES = 128 * BK;      // per CTA: 128 rows of A
 constexpr int P_B_BYTES_MAX = 128 * BK;  // per CTA: up to 128 rows of W
 constexpr int P_STAGE_BYTES = P_A_BYTES + P_B_BYTES_MAX;
+
+constexpr int P_NUM_THREADS = 320;       // 10 warps: producer, MMA issuer, 4 epilogue, 4 activation quantizer
+constexpr int CONV_THREADS = 128;
+constexpr int CONV_ROWS = 4;             // rows of x per quantizer batch; divides 256, so a batch lies in one row block
+constexpr int kMaxRowBlocks = 1024;      // 256-row blocks the in-kernel quantizer can publish (T <= 262144)
+constexpr int kReadySlots = 32;          // concurrently running launches that can each own a set of counters
 
 constexpr int P_OUT_BUF_BYTES = 32 * 128;        // one epilogue warp's staging tile: 32 rows x 64 columns x 2 B
 constexpr int P_OUT_BYTES = 4 * 2 * P_OUT_BUF_BYTES;   // 4 warps, double buffered
@@ -311,6 +327,7 @@ struct PairTail {
     float bias[256];
     uint32_t tmem_base;
     volatile int abort_flag;
+    int is_last_cta;
 };
 
 // the dynamic shared memory window of a CTA without static shared memory starts 1024-byte aligned; the kernel
@@ -319,9 +336,73 @@ constexpr size_t kPairSmemBytes = (size_t)P_STAGES * P_STAGE_BYTES + P_OUT_BYTES
 
 struct PairParams {
     LinearParams lp;
-    int bn;             // tile width in output channels
     int pair_m_blocks;  // ceil(T / 256)
+    int n_tiles;        // column tiles per 256-row block
+    int base_units;     // tile j is (base_units + (j < rem_units)) * 16 columns wide
+    int rem_units;
+    int w_box_rows;     // rows of W each CTA loads per stage: half of the widest tile
+    // in-kernel activation quantizer (x == nullptr: A was quantized by an earlier launch)
+    const uint16_t* x;  // [T, K] 16-bit activations
+    uint8_t* a_int8;    // [T, K] int8 codes (workspace), what tmap_a reads
+    unsigned* ready;    // [pair_m_blocks] rows of each 256-row block that are quantized and visible; zero at launch
+    unsigned* done;     // CTAs that have finished; the last one zeroes `ready` and this counter again
+    float qn, qp;
 };
+
+// first column and width of column tile j
+__host__ __device__ __forceinline__ void pair_tile_cols(const PairParams& pp, int j, int* n0, int* width) {
+    const int extra = j < pp.rem_units ? j : pp.rem_units;
+    *n0 = 16 * (j * pp.base_units + extra);
+    *width = 16 * (pp.base_units + (j < pp.rem_units ? 1 : 0));
+}
+
+// Eq. 1 with the fixed factor on 16 consecutive elements: two 128-bit words of 16-bit values -> one of int8 codes
+template <bool BF>
+__device__ __forceinline__ uint4 quantize16(const uint4& a, const uint4& b, float inv, float qn, float qp) {
+    const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        uint32_t packed = 0;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const float2 f = widen2<BF>(w[2 * q + h]);
+            const int c0 = __float2int_rn(fminf(fmaxf(__fmul_rn(f.x, inv), -qn), qp));
+            const int c1 = __float2int_rn(fminf(fmaxf(__fmul_rn(f.y, inv), -qn), qp));
+            packed |= ((uint32_t)(c0 & 0xFF) | ((uint32_t)(c1 & 0xFF) << 8)) << (16 * h);
+        }
+        o[q] = packed;
+    }
+    return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+__device__ __forceinline__ uint4 ld_stream16(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+// Bounded wait until *counter (written by other CTAs with a fence before their atomic add) reaches `need`.
+__device__ __forceinline__ bool wait_rows_ready(const unsigned* counter, unsigned need, PairTail* tail,
+                                                const LinearParams& p) {
+    const long long t0 = clock64();
+    int polls = 0;
+    for (;;) {
+        unsigned v;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+        if (v >= need) return true;
+        if ((++polls & 15) == 0) {
+            if (tail->abort_flag) return false;
+            if (clock64() - t0 > p.wait_limit) {
+                tail->abort_flag = 1;
+                atomicMax(p.status, (int)SASQ_ERR_TIMEOUT);
+                return false;
+            }
+        }
+        __nanosleep(64);
+    }
+}
 
 __device__ __forceinline__ bool wait_bounded_pair(uint64_t* bar, uint32_t parity, PairTail* tail,
                                                   const LinearParams& p) {
@@ -385,9 +466,7 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();        // 0 = leader
-    const int bn = pp.bn;
-    const int half_bn = bn >> 1;
-    const uint32_t stage_tx = (uint32_t)(P_A_BYTES + half_bn * BK);   // bytes this CTA's two loads deliver
+    const uint32_t stage_tx = (uint32_t)(P_A_BYTES + pp.w_box_rows * BK);   // bytes this CTA's two loads deliver
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < P_STAGES; ++s) {
@@ -415,84 +494,86 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = tail->tmem_base;
 
-    const int n_blocks = (p.N + bn - 1) / bn;
-    const int num_tiles = pp.pair_m_blocks * n_blocks;
+    const int num_tiles = pp.pair_m_blocks * pp.n_tiles;
     const int pair_id = blockIdx.x >> 1;
     const int num_pairs = gridDim.x >> 1;
 
     if (warp == 0) {
         // ---------------- TMA producer (both CTAs) ----------------
-        int stage = 0;
-        uint32_t phase = 0;
-        bool ok = true;
-        for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs) {
-            const int m_blk = tile % pp.pair_m_blocks, n_blk = tile / pp.pair_m_blocks;
-            const int a_row = m_blk * PBM + (int)rank * 128;
-            const int w_row = n_blk * bn + (int)rank * half_bn;
-            for (int kb = 0; kb < p.k_blocks && ok; ++kb) {
-                if (lane == 0) {
+        if (ptx::elect_one()) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs) {
+                const int m_blk = tile % pp.pair_m_blocks;
+                int n0, bn;
+                pair_tile_cols(pp, tile / pp.pair_m_blocks, &n0, &bn);
+                const int a_row = m_blk * PBM + (int)rank * 128;
+                // this CTA's half of the tile's W rows; the box is as high as half the widest tile, so a narrower
+                // tile fetches 8 rows it does not use (rows past N read as zero)
+                const int w_row = n0 + (int)rank * (bn >> 1);
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
                     ok = wait_bounded_pair(&tail->empty[stage], phase ^ 1u, tail, p);
-                    if (ok) {
-                        uint8_t* a_dst = tiles + (size_t)stage * P_STAGE_BYTES;
-                        uint8_t* b_dst = a_dst + P_A_BYTES;
-                        // Only the leader arms the barrier (with the bytes of both CTAs); the partner's copies
-                        // may complete first, which merely drives the transaction count negative for a while:
-                        // the phase cannot complete before the leader's arrival.
-                        const uint32_t full_leader = ptx::mapa_u32(ptx::smem_u32(&tail->full[stage]), 0);
-                        if (rank == 0) ptx::mbar_arrive_expect_tx(&tail->full[stage], 2u * stage_tx);
-                        ptx::tma_load_2d_pair(a_dst, &tmap_a, full_leader, kb * BK, a_row);
-                        ptx::tma_load_2d_pair(b_dst, &tmap_w, full_leader, kb * BK, w_row);
-                    }
+                    if (!ok) break;
+                    uint8_t* a_dst = tiles + (size_t)stage * P_STAGE_BYTES;
+                    uint8_t* b_dst = a_dst + P_A_BYTES;
+                    // Only the leader arms the barrier (with the bytes of both CTAs); the partner's copies
+                    // may complete first, which merely drives the transaction count negative for a while:
+                    // the phase cannot complete before the leader's arrival.
+                    const uint32_t full_leader = ptx::mapa_u32(ptx::smem_u32(&tail->full[stage]), 0);
+                    if (rank == 0) ptx::mbar_arrive_expect_tx(&tail->full[stage], 2u * stage_tx);
+                    ptx::tma_load_2d_pair(a_dst, &tmap_a, full_leader, kb * BK, a_row);
+                    ptx::tma_load_2d_pair(b_dst, &tmap_w, full_leader, kb * BK, w_row);
+                    if (++stage == P_STAGES) { stage = 0; phase ^= 1u; }
                 }
-                ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
-                if (++stage == P_STAGES) { stage = 0; phase ^= 1u; }
+            }
+            // after an abort, copies may still be in flight into this CTA's shared memory: their barrier lives in
+            // the leader, so give them a bounded grace period (a copy takes microseconds) before the CTA may exit
+            if (!ok) {
+                const long long t0 = clock64();
+                while (clock64() - t0 < (1LL << 22)) __nanosleep(1000);
             }
         }
-        // after an abort, copies may still be in flight into this CTA's shared memory: their barrier lives in
-        // the leader, so give them a bounded grace period (a copy takes microseconds) before the CTA may exit
-        if (!ok) {
-            const long long t0 = clock64();
-            while (clock64() - t0 < (1LL << 22)) __nanosleep(1000);
-        }
+        __syncwarp();
     } else if (warp == 1) {
         // ---------------- MMA issuer (leader CTA only) ----------------
-        if (rank == 0) {
-            const uint32_t idesc = ptx::idesc_i8(PBM, bn);
+        if (rank == 0 && ptx::elect_one()) {
+            const uint64_t a_desc0 = ptx::smem_desc_k_major_sw128(ptx::smem_u32(tiles));
+            const uint64_t b_desc0 = ptx::smem_desc_k_major_sw128(ptx::smem_u32(tiles) + P_A_BYTES);
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
             int it = 0;
             for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs, ++it) {
+                int n0, bn;
+                pair_tile_cols(pp, tile / pp.pair_m_blocks, &n0, &bn);
+                const uint32_t idesc = ptx::idesc_i8(PBM, bn);
                 const int buf = it & 1;
                 const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-                if (lane == 0) ok = wait_bounded_pair(&tail->tmem_empty[buf], acc_phase ^ 1u, tail, p);
-                ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
+                ok = wait_bounded_pair(&tail->tmem_empty[buf], acc_phase ^ 1u, tail, p);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 256);
-                for (int kb = 0; kb < p.k_blocks && ok; ++kb) {
-                    if (lane == 0) {
-                        ok = wait_bounded_pair(&tail->full[stage], phase, tail, p);
-                        if (ok) {
-                            ptx::tc_fence_after_sync();
-                            const uint32_t a_addr = ptx::smem_u32(tiles + (size_t)stage * P_STAGE_BYTES);
-                            const uint64_t a_desc = ptx::smem_desc_k_major_sw128(a_addr);
-                            const uint64_t b_desc = ptx::smem_desc_k_major_sw128(a_addr + P_A_BYTES);
-#pragma unroll
-                            for (int k = 0; k < BK / UMMA_K; ++k) {
-                                ptx::mma_i8_ss_pair(d_tmem, a_desc + (uint64_t)(k * (UMMA_K >> 4)),
-                                                    b_desc + (uint64_t)(k * (UMMA_K >> 4)), idesc,
-                                                    (kb | k) != 0 ? 1u : 0u);
-                            }
-                            ptx::mma_commit_pair(&tail->empty[stage], 0x3);
-                            if (kb == p.k_blocks - 1) ptx::mma_commit_pair(&tail->tmem_full[buf], 0x3);
-                        }
-                    }
-                    ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
+                uint32_t accumulate = 0;            // the first MMA of a tile overwrites the accumulators
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    ok = wait_bounded_pair(&tail->full[stage], phase, tail, p);
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
+                    // 32 bytes of K per MMA inside the swizzled 128-byte row: +2 in the descriptor's address field
+                    const uint64_t a_desc = a_desc0 + (uint64_t)(stage * (P_STAGE_BYTES >> 4));
+                    const uint64_t b_desc = b_desc0 + (uint64_t)(stage * (P_STAGE_BYTES >> 4));
+                    ptx::mma_i8_ss_pair(d_tmem, a_desc, b_desc, idesc, accumulate);
+                    ptx::mma_i8_ss_pair_acc(d_tmem, a_desc + 2, b_desc + 2, idesc);
+                    ptx::mma_i8_ss_pair_acc(d_tmem, a_desc + 4, b_desc + 4, idesc);
+                    ptx::mma_i8_ss_pair_acc(d_tmem, a_desc + 6, b_desc + 6, idesc);
+                    accumulate = 1u;
+                    ptx::mma_commit_pair(&tail->empty[stage], 0x3);          // stage reusable once these MMAs are done
+                    if (kb == p.k_blocks - 1) ptx::mma_commit_pair(&tail->tmem_full[buf], 0x3);
                     if (++stage == P_STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
         }
+        __syncwarp();
     } else {
         // ---------------- epilogue (warps 2..5 of both CTAs) ----------------
         const int quad = warp & 3;
@@ -504,10 +585,11 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         int it = 0;
         unsigned out_flip = 0;
         for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs, ++it) {
-            const int m_blk = tile % pp.pair_m_blocks, n_blk = tile / pp.pair_m_blocks;
+            const int m_blk = tile % pp.pair_m_blocks;
+            int n0, bn;
+            pair_tile_cols(pp, tile / pp.pair_m_blocks, &n0, &bn);
             const int buf = it & 1;
             const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-            const int n0 = n_blk * bn;
             asm volatile("bar.sync 1, 128;" ::: "memory");
             for (int j = et; j < bn; j += EPI_THREADS) {
                 const int n = n0 + j;
@@ -644,24 +726,8 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const uint4* __restri
                                                            float qn, float qp) {
     const float inv = __fdiv_rn(1.0f, __ldg(x_scale));
     const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += stride) {
-        const uint4 a = x[2 * i], b = x[2 * i + 1];
-        const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-        uint32_t o[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            uint32_t packed = 0;
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const float2 f = widen2<BF>(w[2 * q + h]);
-                const int c0 = __float2int_rn(fminf(fmaxf(__fmul_rn(f.x, inv), -qn), qp));
-                const int c1 = __float2int_rn(fminf(fmaxf(__fmul_rn(f.y, inv), -qn), qp));
-                packed |= ((uint32_t)(c0 & 0xFF) | ((uint32_t)(c1 & 0xFF) << 8)) << (16 * h);
-            }
-            o[q] = packed;
-        }
-        out[i] = make_uint4(o[0], o[1], o[2], o[3]);
-    }
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += stride)
+        out[i] = quantize16<BF>(x[2 * i], x[2 * i + 1], inv, qn, qp);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -773,17 +839,28 @@ int pair_capacity(bool bf, int sm_count) {
     return clusters;
 }
 
-// Tile width (multiple of 16, 128..256) that minimises waves x width for this problem on `pairs` CTA pairs.
-int choose_bn(int pair_m_blocks, int N, int pairs) {
-    int best = 256;
-    long long best_cost = -1;
-    for (int bn = 256; bn >= 128; bn -= 16) {
-        const long long tiles = (long long)pair_m_blocks * ((N + bn - 1) / bn);
-        const long long waves = (tiles + pairs - 1) / pairs;
-        const long long cost = waves * bn;
-        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = bn; }
+// Column tiling of a 256-row block for `pairs` resident CTA pairs.  One MMA of N columns keeps the tensor pipe
+// busy for about max(N, 208) / 2 cycles (below 208 columns the instruction is bound by reading its A operand), and a
+// launch takes as long as its fullest pair: waves x that cost of the widest tile.  Tiles are at least 16 x 8 = 128
+// columns wide unless N itself is narrower.  Fewer, wider tiles win ties (less fixed work per tile).
+void plan_pair_tiles(PairParams* pp, int m_blocks, long long N, int pairs) {
+    const int units = (int)((N + 15) / 16);
+    int best_nt = (units + 15) / 16;
+    double best_cost = -1.0;
+    for (int nt = (units + 15) / 16; nt <= units; ++nt) {
+        const int base = units / nt, rem = units % nt;
+        const int max_w = 16 * (base + (rem ? 1 : 0));
+        if (max_w > 256) continue;
+        if (max_w < 128 && nt > (units + 15) / 16) break;
+        const long long waves = ((long long)m_blocks * nt + pairs - 1) / pairs;
+        const double cost = (double)waves * (max_w > 208 ? max_w : 208);
+        if (best_cost < 0.0 || cost < 0.99 * best_cost) { best_cost = cost; best_nt = nt; }
     }
-    return best;
+    pp->pair_m_blocks = m_blocks;
+    pp->n_tiles = best_nt;
+    pp->base_units = units / best_nt;
+    pp->rem_units = units % best_nt;
+    pp->w_box_rows = 8 * (pp->base_units + (pp->rem_units ? 1 : 0));
 }
 
 int* status_word_ptr() {
@@ -816,6 +893,26 @@ bool single_kernel_ready(bool bf) {
 }  // namespace sasq
 
 extern "C" {
+
+int sasq_static_w8a8_linear_tiles(int64_t T, int64_t N, int num_pairs, int pair_id, int32_t* tiles_host, int cap) {
+    using namespace sasq;
+    if (T <= 0 || N <= 0 || T > (1 << 24) || N > (1 << 24) || num_pairs <= 0 || pair_id < 0 || pair_id >= num_pairs ||
+        cap < 0 || (cap > 0 && tiles_host == nullptr))
+        return -1;
+    PairParams pp{};
+    plan_pair_tiles(&pp, (int)((T + PBM - 1) / PBM), N, num_pairs);
+    const int num_tiles = pp.pair_m_blocks * pp.n_tiles;
+    int n = 0;
+    for (int tile = pair_id; tile < num_tiles; tile += num_pairs, ++n) {
+        if (n >= cap) continue;
+        int n0, width;
+        pair_tile_cols(pp, tile / pp.pair_m_blocks, &n0, &width);
+        tiles_host[3 * n + 0] = (tile % pp.pair_m_blocks) * PBM;
+        tiles_host[3 * n + 1] = n0;
+        tiles_host[3 * n + 2] = width;
+    }
+    return n;
+}
 
 size_t sasq_static_w8a8_linear_workspace(int64_t T, int64_t N, int64_t K) {
     (void)N;
@@ -878,16 +975,15 @@ int sasq_static_w8a8_linear(const void* x, const int8_t* w, const float* w_scale
     CUtensorMap tmap_a, tmap_w;
     cudaError_t e;
     if (T > BM) {
-        // CTA pairs, 256 x bn tiles; bn minimises (waves x bn) over the resident pairs
+        // CTA pairs, 256-row blocks cut into evenly wide column tiles that fill whole waves of the resident pairs
         const int pairs = pair_capacity(dt == SASQ_BF16, sm_count);
         if (pairs <= 0) return SASQ_ERR_CUDA;
         PairParams pp{};
-        pp.pair_m_blocks = (int)((T + PBM - 1) / PBM);
-        pp.bn = choose_bn(pp.pair_m_blocks, (int)N, pairs);
+        plan_pair_tiles(&pp, (int)((T + PBM - 1) / PBM), N, pairs);
         p.m_blocks = pp.pair_m_blocks;
-        p.n_blocks = (int)((N + pp.bn - 1) / pp.bn);
+        p.n_blocks = pp.n_tiles;
         pp.lp = p;
-        if (!make_tmap(&tmap_a, a_int8, T, K, 128) || !make_tmap(&tmap_w, w, N, K, pp.bn / 2)) return SASQ_ERR_CUDA;
+        if (!make_tmap(&tmap_a, a_int8, T, K, 128) || !make_tmap(&tmap_w, w, N, K, pp.w_box_rows)) return SASQ_ERR_CUDA;
         CUtensorMap tmap_y64, tmap_y16;
         if (!make_tmap_out(&tmap_y64, y, T, N, 64) || !make_tmap_out(&tmap_y16, y, T, N, 16)) return SASQ_ERR_CUDA;
         const long long tiles = (long long)p.m_blocks * p.n_blocks;
