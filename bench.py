@@ -162,17 +162,18 @@ class Layer:
         torch.cuda.synchronize()
         assert P.sasq_device_status() == 0
 
-    # kernels launched per step: fused quantizer + combine, then (quantize-on-load is inside the linear call)
+    # kernels launched per step: one fused quantizer launch (the reduction's second stage runs in its last block),
+    # then one launch per linear (its activation quantizer runs inside the GEMM kernel)
     def phase_a(self):
         self.P.sasq_fakequant_fwd_bwd_multi(self.descs, self.scales, self.grads, self.q_ws, BITS)
-        return 2
+        return 1
 
     def phase_b(self):
         n = 0
         for i in range(7):
             self.P.sasq_static_w8a8_linear(self.x[i], self.w_int[i], self.w_scale[i], self.scales[i:i + 1],
                                            self.out[i], workspace=self.l_ws, bits=BITS)
-            n += self.P.LAUNCHES_PER_LINEAR
+            n += self.P.linear_launches(T_TOKENS)
         return n
 
 

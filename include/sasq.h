@@ -170,7 +170,7 @@ SASQ_API int sasq_static_w8a8_linear(const void* x, const int8_t* w, const float
 /* How sasq_static_w8a8_linear splits a [T, N] output over `num_pairs` co-operating CTA pairs when T > 128
  * (introspection for tests and tuning; runs on the host, touches no device).  Every 256-row block is cut into the
  * same number of column tiles, widths multiples of 16 that differ by at most 16; the number is chosen so that the
- * tiles fill whole waves of the pairs; tile t goes to pair t % num_pairs, row blocks fastest.  Writes up to `cap`
+ * tiles fill whole waves of the pairs; tile t goes to pair t % num_pairs, column tiles fastest.  Writes up to `cap`
  * triples (first row, first column, width in columns) of pair `pair_id` to tiles_host (HOST memory, [cap][3]
  * int32) and returns how many tiles the pair has, or -1 for invalid arguments. */
 SASQ_API int sasq_static_w8a8_linear_tiles(int64_t T, int64_t N, int num_pairs, int pair_id, int32_t* tiles_host,

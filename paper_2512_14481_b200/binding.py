@@ -18,13 +18,18 @@ __all__ = [
     "sasq_fakequant_fwd", "sasq_fakequant_bwd_workspace", "sasq_fakequant_bwd", "sasq_fakequant_fwd_bwd",
     "sasq_fakequant_multi_workspace", "sasq_fakequant_fwd_bwd_multi", "sasq_static_w8a8_linear_workspace",
     "sasq_static_w8a8_linear", "sasq_device_status", "QDesc", "sasq_absmax_scale_workspace", "sasq_absmax_scale",
-    "sasq_quantize_weight", "LAUNCHES_PER_LINEAR", "sasq_fakequant_fwd_bwd_static", "sasq_static_w8a8_linear_tiles",
+    "sasq_quantize_weight", "linear_launches", "sasq_fakequant_fwd_bwd_static", "sasq_static_w8a8_linear_tiles",
 ]
 
 SASQ_F16 = 0
 SASQ_BF16 = 1
-# kernels one sasq_static_w8a8_linear call launches (activation quantizer + GEMM); used to count launches
-LAUNCHES_PER_LINEAR = 2
+
+
+def linear_launches(T: int) -> int:
+    """Kernels one sasq_static_w8a8_linear call launches, for launch counting: one when the activation quantizer
+    runs inside the GEMM kernel (128 < T <= 262144), otherwise the quantizer and the GEMM."""
+    return 1 if 128 < int(T) <= 262144 else 2
+
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libsasq_b200.so")

@@ -32,6 +32,19 @@ namespace sasq {
         return h;                                                                            \
     }
 
+// ---------------------------------------------------------------------------
+// Programmatic dependent launch.  The hot kernels are launched with the
+// programmatic-stream-serialization attribute: the next kernel of the stream may
+// be scheduled while this one still runs (as SMs free up) and does its set-up,
+// then waits here until every kernel before it has completed and its memory is
+// visible.  Nothing that an earlier kernel may have written (or may still read)
+// is touched before pdl_wait().  Without the attribute both are no-ops.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void pdl_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ bool scale_is_bad(float s) {
     const float inv = __fdiv_rn(1.0f, s);
     return !(s == s) || s == 0.0f || isinf(s) || isinf(inv) || !(inv == inv);
@@ -83,6 +96,14 @@ __device__ __forceinline__ uint16_t narrow1(float f) {
 // host-side checks
 // ---------------------------------------------------------------------------
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// launch attribute that lets a kernel start its set-up under the tail of the kernel before it in the stream
+inline cudaLaunchAttribute pdl_attribute() {
+    cudaLaunchAttribute a{};
+    a.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    a.val.programmaticStreamSerializationAllowed = 1;
+    return a;
+}
 
 // SM count of the current device if it is sm_100 (compute capability 10.x), else <= 0.
 int device_sm_count_if_sm100();

@@ -51,9 +51,14 @@ unsigned* next_ticket() {
 
 template <bool BF, bool FWD, bool BWD>
 cudaError_t launch_stream(const QParams& p, int grid, cudaStream_t st) {
-    fakequant_kernel<BF, FWD, BWD, kThreads, kUnroll, kBlocksPerSM, kLoadHint, kStoreHint>
-        <<<grid, kThreads, 0, st>>>(p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1] = {pdl_attribute()};
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, fakequant_kernel<BF, FWD, BWD, kThreads, kUnroll, kBlocksPerSM, kLoadHint, kStoreHint>, p);
 }
 
 template <bool BF>

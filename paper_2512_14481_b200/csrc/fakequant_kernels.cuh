@@ -122,6 +122,8 @@ __device__ __forceinline__ double block_sum_fixed(double v, double* smem /* [THR
 template <bool BF, bool FWD, bool BWD, int THREADS, int UNROLL, int MIN_BLOCKS, int LHINT, int SHINT>
 __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) fakequant_kernel(const __grid_constant__ QParams p) {
     __shared__ double warp_sums[THREADS / 32];
+    pdl_launch_dependents();
+    pdl_wait();
     const float qn = p.qn, qp = p.qp;
     const long long gtid = (long long)blockIdx.x * THREADS + threadIdx.x;
     const long long gstride = (long long)gridDim.x * THREADS;

@@ -7,11 +7,12 @@
 //   warp 0      TMA producer: W tiles and int8 A tiles -> 128-byte-swizzled shared memory
 //   warp 1      MMA issuer: tcgen05.mma.kind::i8, 32 bytes of K per instruction, TMEM double-buffered
 //   warps 2..5  epilogue: tcgen05.ld -> dequant -> 16-bit stores, overlapped with the next tile's mainloop
-//   warps 6..9  (CTA-pair kernel) activation quantizer: Eq. 1 with the fixed factor on rows of x -> int8 A in the
+//   warps 6..13 (CTA-pair kernel) activation quantizer: Eq. 1 with the fixed factor on rows of x -> int8 A in the
 //               workspace, published per 256-row block; the producers wait for the block they are about to load,
 //               so the quantization of later rows runs under the MMAs of earlier ones and costs no launch
 // Every wait on an mbarrier is bounded; a wait that gives up raises SASQ_ERR_TIMEOUT
 // in the sticky status word and all roles fall through to the teardown.
+#include <atomic>
 #include <mutex>
 
 #include "common.cuh"
@@ -309,9 +310,10 @@ constexpr int P_A_BYTES = 128 * BK;      // per CTA: 128 rows of A
 constexpr int P_B_BYTES_MAX = 128 * BK;  // per CTA: up to 128 rows of W
 constexpr int P_STAGE_BYTES = P_A_BYTES + P_B_BYTES_MAX;
 
-constexpr int P_NUM_THREADS = 320;       // 10 warps: producer, MMA issuer, 4 epilogue, 4 activation quantizer
-constexpr int CONV_THREADS = 128;
-constexpr int CONV_ROWS = 4;             // rows of x per quantizer batch; divides 256, so a batch lies in one row block
+constexpr int P_NUM_THREADS = 448;       // 14 warps: producer, MMA issuer, 4 epilogue, 8 activation quantizer
+constexpr int CONV_THREADS = 256;
+constexpr int CONV_ITEMS = 16;           // 8-element items per thread and chunk: 16 128-bit loads in flight per thread
+constexpr int CONV_CHUNK = CONV_THREADS * CONV_ITEMS;   // items per chunk (32768 elements)
 constexpr int kMaxRowBlocks = 1024;      // 256-row blocks the in-kernel quantizer can publish (T <= 262144)
 constexpr int kReadySlots = 32;          // concurrently running launches that can each own a set of counters
 
@@ -344,7 +346,7 @@ struct PairParams {
     // in-kernel activation quantizer (x == nullptr: A was quantized by an earlier launch)
     const uint16_t* x;  // [T, K] 16-bit activations
     uint8_t* a_int8;    // [T, K] int8 codes (workspace), what tmap_a reads
-    unsigned* ready;    // [pair_m_blocks] rows of each 256-row block that are quantized and visible; zero at launch
+    unsigned* ready;    // [pair_m_blocks] 8-element items of each 256-row block that are quantized and visible; zero at launch
     unsigned* done;     // CTAs that have finished; the last one zeroes `ready` and this counter again
     float qn, qp;
 };
@@ -356,24 +358,34 @@ __host__ __device__ __forceinline__ void pair_tile_cols(const PairParams& pp, in
     *width = 16 * (pp.base_units + (j < pp.rem_units ? 1 : 0));
 }
 
-// Eq. 1 with the fixed factor on 16 consecutive elements: two 128-bit words of 16-bit values -> one of int8 codes
-template <bool BF>
-__device__ __forceinline__ uint4 quantize16(const uint4& a, const uint4& b, float inv, float qn, float qp) {
-    const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-    uint32_t o[4];
+// Eq. 1 with the fixed factor on 8 consecutive elements: one 128-bit word of 16-bit values -> 8 int8 codes.
+//   t = x * fl32(1/s) (one fp32 multiply);  code = clamp(rint(t), -Qn, Qp).
+// fmax first: it maps NaN to -Qn (the documented behaviour) and applies the lower clamp.  With 8 bits the upper
+// clamp and the rounding are what the saturating round-to-nearest-even conversion to s32 followed by the
+// saturating pack to s8 does anyway (Qn = 128, Qp = 127); narrower codes take an fmin as well.
+template <bool BF, bool EIGHT_BITS>
+__device__ __forceinline__ uint2 quantize8(const uint4& v, float inv, float qn, float qp) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    int c[8];
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-        uint32_t packed = 0;
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const float2 f = widen2<BF>(w[2 * q + h]);
-            const int c0 = __float2int_rn(fminf(fmaxf(__fmul_rn(f.x, inv), -qn), qp));
-            const int c1 = __float2int_rn(fminf(fmaxf(__fmul_rn(f.y, inv), -qn), qp));
-            packed |= ((uint32_t)(c0 & 0xFF) | ((uint32_t)(c1 & 0xFF) << 8)) << (16 * h);
+        const float2 f = widen2<BF>(w[q]);
+        float t0 = fmaxf(__fmul_rn(f.x, inv), -qn);
+        float t1 = fmaxf(__fmul_rn(f.y, inv), -qn);
+        if constexpr (!EIGHT_BITS) {
+            t0 = fminf(t0, qp);
+            t1 = fminf(t1, qp);
         }
-        o[q] = packed;
+        c[2 * q] = __float2int_rn(t0);          // saturates at the int32 range
+        c[2 * q + 1] = __float2int_rn(t1);
     }
-    return make_uint4(o[0], o[1], o[2], o[3]);
+    uint32_t lo, hi, t;
+    // cvt.pack.sat.s8.s32.b32 d, a, b, c:  d = (sat8(a) << 8 | sat8(b)) | (c << 16)
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(t) : "r"(c[3]), "r"(c[2]), "r"(0));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(lo) : "r"(c[1]), "r"(c[0]), "r"(t));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(t) : "r"(c[7]), "r"(c[6]), "r"(0));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(c[5]), "r"(c[4]), "r"(t));
+    return make_uint2(lo, hi);
 }
 
 __device__ __forceinline__ uint4 ld_stream16(const uint4* p) {
@@ -449,7 +461,7 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t* v, const float* s
 }
 
 template <bool BF>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(P_NUM_THREADS, 1)
 w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                       const __grid_constant__ CUtensorMap tmap_y64, const __grid_constant__ CUtensorMap tmap_y16,
                       const __grid_constant__ PairParams pp) {
@@ -462,6 +474,8 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         if (threadIdx.x == 0) atomicMax(p.status, (int)SASQ_ERR_CUDA);
         return;
     }
+
+    pdl_launch_dependents();
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -493,6 +507,7 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     ptx::cluster_sync_all();            // both CTAs' barriers exist before anyone signals across the pair
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = tail->tmem_base;
+    pdl_wait();                         // set-up done; from here on global memory of earlier kernels is used
 
     const int num_tiles = pp.pair_m_blocks * pp.n_tiles;
     const int pair_id = blockIdx.x >> 1;
@@ -504,11 +519,21 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
+            int ready_blk = -1;
             for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs) {
-                const int m_blk = tile % pp.pair_m_blocks;
+                const int m_blk = tile / pp.n_tiles;
                 int n0, bn;
-                pair_tile_cols(pp, tile / pp.pair_m_blocks, &n0, &bn);
+                pair_tile_cols(pp, tile - m_blk * pp.n_tiles, &n0, &bn);
                 const int a_row = m_blk * PBM + (int)rank * 128;
+                if (pp.x != nullptr && m_blk != ready_blk) {
+                    // the rows of this block must have been quantized, by whichever CTAs had them, and be visible
+                    // to the TMA unit before the first load of the tile
+                    const int rows = p.T - m_blk * PBM;
+                    ok = wait_rows_ready(pp.ready + m_blk, (unsigned)((rows < PBM ? rows : PBM) * (p.K >> 3)), tail, p);
+                    if (!ok) break;
+                    asm volatile("fence.proxy.async.global;" ::: "memory");
+                    ready_blk = m_blk;
+                }
                 // this CTA's half of the tile's W rows; the box is as high as half the widest tile, so a narrower
                 // tile fetches 8 rows it does not use (rows past N read as zero)
                 const int w_row = n0 + (int)rank * (bn >> 1);
@@ -546,7 +571,7 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             int it = 0;
             for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs, ++it) {
                 int n0, bn;
-                pair_tile_cols(pp, tile / pp.pair_m_blocks, &n0, &bn);
+                pair_tile_cols(pp, tile % pp.n_tiles, &n0, &bn);
                 const uint32_t idesc = ptx::idesc_i8(PBM, bn);
                 const int buf = it & 1;
                 const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
@@ -574,6 +599,72 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             }
         }
         __syncwarp();
+    } else if (warp >= 6) {
+        // ---------------- activation quantizer (warps 6..13 of both CTAs) ----------------
+        // x is taken as a flat run of T * K / 8 items of 8 elements, cut into chunks that are dealt round-robin
+        // over the CTAs in address order, so the row blocks become ready in the order the tiles need them.  Each
+        // thread keeps 16 128-bit loads in flight; the loads of a CTA's next chunk are issued before the fence and
+        // barrier that publish the current one, so their latencies overlap.
+        if (pp.x != nullptr) {
+            const int ct = threadIdx.x - (P_NUM_THREADS - CONV_THREADS);
+            const float inv = __fdiv_rn(1.0f, __ldg(p.x_scale));
+            const float qn = pp.qn, qp = pp.qp;
+            const bool eight = qp == 127.0f;
+            const long long items_per_block = (long long)PBM * (p.K >> 3);
+            const long long total = (long long)p.T * (p.K >> 3);
+            const long long n_chunks = (total + CONV_CHUNK - 1) / CONV_CHUNK;
+            const uint4* src = reinterpret_cast<const uint4*>(pp.x);
+            uint2* dst = reinterpret_cast<uint2*>(pp.a_int8);
+            uint4 v[CONV_ITEMS];
+            long long c = blockIdx.x;
+            if (c < n_chunks) {
+#pragma unroll
+                for (int u = 0; u < CONV_ITEMS; ++u) {
+                    const long long i = c * CONV_CHUNK + u * CONV_THREADS + ct;
+                    if (i < total) v[u] = ld_stream16(src + i);
+                }
+            }
+            while (c < n_chunks) {
+                if (eight) {
+#pragma unroll
+                    for (int u = 0; u < CONV_ITEMS; ++u) {
+                        const long long i = c * CONV_CHUNK + u * CONV_THREADS + ct;
+                        if (i < total) dst[i] = quantize8<BF, true>(v[u], inv, qn, qp);
+                    }
+                } else {
+#pragma unroll
+                    for (int u = 0; u < CONV_ITEMS; ++u) {
+                        const long long i = c * CONV_CHUNK + u * CONV_THREADS + ct;
+                        if (i < total) dst[i] = quantize8<BF, false>(v[u], inv, qn, qp);
+                    }
+                }
+                const long long cn = c + gridDim.x;
+                if (cn < n_chunks) {
+#pragma unroll
+                    for (int u = 0; u < CONV_ITEMS; ++u) {
+                        const long long i = cn * CONV_CHUNK + u * CONV_THREADS + ct;
+                        if (i < total) v[u] = ld_stream16(src + i);
+                    }
+                }
+                asm volatile("fence.proxy.async.global;" ::: "memory");
+                __threadfence();
+                asm volatile("bar.sync 3, 256;" ::: "memory");
+                if (ct == 0) {
+                    // credit the chunk's items to the row block(s) they lie in
+                    const long long first = c * CONV_CHUNK;
+                    const long long end = (first + CONV_CHUNK < total) ? first + CONV_CHUNK : total;
+                    long long i = first;
+                    while (i < end) {
+                        const long long blk = i / items_per_block;
+                        const long long blk_end = (blk + 1) * items_per_block;
+                        const long long upto = blk_end < end ? blk_end : end;
+                        atomicAdd(pp.ready + blk, (unsigned)(upto - i));
+                        i = upto;
+                    }
+                }
+                c = cn;
+            }
+        }
     } else {
         // ---------------- epilogue (warps 2..5 of both CTAs) ----------------
         const int quad = warp & 3;
@@ -585,9 +676,9 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         int it = 0;
         unsigned out_flip = 0;
         for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs, ++it) {
-            const int m_blk = tile % pp.pair_m_blocks;
+            const int m_blk = tile / pp.n_tiles;
             int n0, bn;
-            pair_tile_cols(pp, tile / pp.pair_m_blocks, &n0, &bn);
+            pair_tile_cols(pp, tile - m_blk * pp.n_tiles, &n0, &bn);
             const int buf = it & 1;
             const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
             asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -716,18 +807,29 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc_pair(tmem_base, TMEM_COLS);
     }
+    if (pp.x != nullptr) {
+        // the CTA that finishes last leaves the counters at zero for the next launch that draws them
+        if (threadIdx.x == 0) tail->is_last_cta = (atomicAdd(pp.done, 1u) == gridDim.x - 1) ? 1 : 0;
+        __syncthreads();
+        if (tail->is_last_cta) {
+            for (int i = threadIdx.x; i < pp.pair_m_blocks; i += P_NUM_THREADS) pp.ready[i] = 0u;
+            if (threadIdx.x == 0) *pp.done = 0u;
+        }
+    }
 }
 
 // Eq. 1 with the fixed factor, written once to int8 (operand A of the GEMM).
 // 16 elements per thread: two 128-bit loads, one 128-bit store.
+// The same quantizer as a launch of its own (small T, or more row blocks than the in-kernel counters hold):
+// 8 elements per thread and step, one 128-bit load, one 64-bit store.
 template <bool BF>
-__global__ void __launch_bounds__(256) quantize_act_kernel(const uint4* __restrict__ x, uint4* __restrict__ out,
-                                                           long long n16, const float* __restrict__ x_scale,
+__global__ void __launch_bounds__(256) quantize_act_kernel(const uint4* __restrict__ x, uint2* __restrict__ out,
+                                                           long long n8, const float* __restrict__ x_scale,
                                                            float qn, float qp) {
     const float inv = __fdiv_rn(1.0f, __ldg(x_scale));
     const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += stride)
-        out[i] = quantize16<BF>(x[2 * i], x[2 * i + 1], inv, qn, qp);
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += stride)
+        out[i] = quantize8<BF, false>(x[i], inv, qn, qp);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -811,6 +913,31 @@ bool make_tmap_out(CUtensorMap* m, const void* base, long long T, long long N, i
     return make_tmap_generic(m, base, T, N, 32, box_cols, 2);
 }
 
+// Counters of the in-kernel activation quantizer.  They are zero when the library is loaded and every launch leaves
+// the set it used at zero again; launches draw the sets round-robin, so two launches share one only if more than
+// kReadySlots launches of this kernel were running at the same time.
+static __device__ unsigned g_a_ready[kReadySlots][kMaxRowBlocks];
+static __device__ unsigned g_a_done[kReadySlots];
+
+bool next_ready_slot(unsigned** ready, unsigned** done) {
+    static unsigned* ready_base[64] = {nullptr};
+    static unsigned* done_base[64] = {nullptr};
+    static std::atomic<unsigned> next{0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    if (ready_base[dev] == nullptr) {
+        unsigned *r = nullptr, *d = nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&r), g_a_ready) != cudaSuccess) return false;
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&d), g_a_done) != cudaSuccess) return false;
+        done_base[dev] = d;
+        ready_base[dev] = r;
+    }
+    const unsigned slot = next.fetch_add(1u, std::memory_order_relaxed) % kReadySlots;
+    *ready = ready_base[dev] + (size_t)slot * kMaxRowBlocks;
+    *done = done_base[dev] + slot;
+    return true;
+}
+
 // Number of CTA pairs that can be resident at once (one pair per TPC); also opts the kernel in to its shared memory.
 int pair_capacity(bool bf, int sm_count) {
     static int cache[64][2] = {};
@@ -823,7 +950,7 @@ int pair_capacity(bool bf, int sm_count) {
         return -1;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)sm_count, 1, 1);
-    cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+    cfg.blockDim = dim3(P_NUM_THREADS, 1, 1);
     cfg.dynamicSmemBytes = kPairSmemBytes;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -906,8 +1033,8 @@ int sasq_static_w8a8_linear_tiles(int64_t T, int64_t N, int num_pairs, int pair_
     for (int tile = pair_id; tile < num_tiles; tile += num_pairs, ++n) {
         if (n >= cap) continue;
         int n0, width;
-        pair_tile_cols(pp, tile / pp.pair_m_blocks, &n0, &width);
-        tiles_host[3 * n + 0] = (tile % pp.pair_m_blocks) * PBM;
+        pair_tile_cols(pp, tile % pp.n_tiles, &n0, &width);
+        tiles_host[3 * n + 0] = (tile / pp.n_tiles) * PBM;
         tiles_host[3 * n + 1] = n0;
         tiles_host[3 * n + 2] = width;
     }
@@ -943,20 +1070,22 @@ int sasq_static_w8a8_linear(const void* x, const int8_t* w, const float* w_scale
     if (status == nullptr) return SASQ_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
-    // 1. Eq. 1 with the fixed factor -> int8 activations in the workspace
+    // 1. Eq. 1 with the fixed factor -> int8 activations in the workspace: inside the CTA-pair kernel when it is
+    //    used and the row blocks fit its counters, otherwise by a launch of its own
     uint8_t* a_int8 = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(workspace) + 127) & ~uintptr_t(127));
-    const long long n16 = (T * K) / 16;     // K % 16 == 0
     const float qn = (float)(1 << (bits - 1)), qp = (float)((1 << (bits - 1)) - 1);
-    {
-        long long blocks = (n16 + 255) / 256;
+    const bool in_kernel_quantizer = T > BM && (T + PBM - 1) / PBM <= kMaxRowBlocks;
+    if (!in_kernel_quantizer) {
+        const long long n8 = (T * K) / 8;     // K % 16 == 0
+        long long blocks = (n8 + 255) / 256;
         if (blocks > (long long)sm_count * 8) blocks = (long long)sm_count * 8;
         if (dt == SASQ_BF16)
             quantize_act_kernel<true><<<(int)blocks, 256, 0, st>>>(static_cast<const uint4*>(x),
-                                                                   reinterpret_cast<uint4*>(a_int8), n16,
+                                                                   reinterpret_cast<uint2*>(a_int8), n8,
                                                                    x_scale_dev, qn, qp);
         else
             quantize_act_kernel<false><<<(int)blocks, 256, 0, st>>>(static_cast<const uint4*>(x),
-                                                                    reinterpret_cast<uint4*>(a_int8), n16,
+                                                                    reinterpret_cast<uint2*>(a_int8), n8,
                                                                     x_scale_dev, qn, qp);
         if (cudaGetLastError() != cudaSuccess) return SASQ_ERR_CUDA;
     }
@@ -983,6 +1112,13 @@ int sasq_static_w8a8_linear(const void* x, const int8_t* w, const float* w_scale
         p.m_blocks = pp.pair_m_blocks;
         p.n_blocks = pp.n_tiles;
         pp.lp = p;
+        pp.qn = qn;
+        pp.qp = qp;
+        if (in_kernel_quantizer) {
+            pp.x = static_cast<const uint16_t*>(x);
+            pp.a_int8 = a_int8;
+            if (!next_ready_slot(&pp.ready, &pp.done)) return SASQ_ERR_CUDA;
+        }
         if (!make_tmap(&tmap_a, a_int8, T, K, 128) || !make_tmap(&tmap_w, w, N, K, pp.w_box_rows)) return SASQ_ERR_CUDA;
         CUtensorMap tmap_y64, tmap_y16;
         if (!make_tmap_out(&tmap_y64, y, T, N, 64) || !make_tmap_out(&tmap_y16, y, T, N, 16)) return SASQ_ERR_CUDA;
@@ -990,16 +1126,17 @@ int sasq_static_w8a8_linear(const void* x, const int8_t* w, const float* w_scale
         const int grid = 2 * (int)(tiles < pairs ? tiles : pairs);
         cudaLaunchConfig_t cfg{};
         cfg.gridDim = dim3((unsigned)grid, 1, 1);
-        cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+        cfg.blockDim = dim3(P_NUM_THREADS, 1, 1);
         cfg.dynamicSmemBytes = kPairSmemBytes;
         cfg.stream = st;
-        cudaLaunchAttribute attr[1];
+        cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = 2;
         attr[0].val.clusterDim.y = 1;
         attr[0].val.clusterDim.z = 1;
+        attr[1] = pdl_attribute();
         cfg.attrs = attr;
-        cfg.numAttrs = 1;
+        cfg.numAttrs = 2;
         if (dt == SASQ_BF16) e = cudaLaunchKernelEx(&cfg, w8a8_gemm_pair_kernel<true>, tmap_a, tmap_w, tmap_y64, tmap_y16, pp);
         else e = cudaLaunchKernelEx(&cfg, w8a8_gemm_pair_kernel<false>, tmap_a, tmap_w, tmap_y64, tmap_y16, pp);
         if (e != cudaSuccess) return SASQ_ERR_CUDA;
