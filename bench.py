@@ -69,6 +69,8 @@ def linear_ops():
 # clocks during the timed region (NVML, read-only)
 # ---------------------------------------------------------------------------
 class ClockSampler:
+    PERIOD_S = 0.005
+
     REASONS = {
         0x0000000000000004: "sw_power_cap",
         0x0000000000000008: "hw_slowdown",
@@ -101,7 +103,7 @@ class ClockSampler:
                         self.reasons.add(name)
             except Exception:
                 pass
-            self._stop.wait(0.02)
+            self._stop.wait(self.PERIOD_S)
 
     def start(self):
         if self._nv is not None:
@@ -177,6 +179,19 @@ class Layer:
         return n
 
 
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of per-rank timings (the slowest rank decides); identity without a process group."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
+
+
+def throughput(world: int, units_per_rank: float, steps: int, ms: float) -> float:
+    """Whole-job rate: the units all ranks processed over the slowest rank's time (weak scaling, replicas)."""
+    return world * units_per_rank * steps / (ms * 1e-3)
+
+
 def run_ours(args):
     import paper_2512_14481_b200 as P          # raises if the CUDA library has not been built: no fallback
 
@@ -228,10 +243,7 @@ def run_ours(args):
     ms_a = sum(ev[k][0].elapsed_time(ev[k][1]) for k in range(K))
     ms_b = sum(ev[k][1].elapsed_time(ev[k][2]) for k in range(K))
     ms_total = ev[0][0].elapsed_time(ev[K - 1][2])
-    times = torch.tensor([ms_a, ms_b, ms_total], dtype=torch.float64, device=device)
-    if dist is not None:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_a, ms_b, ms_total = [float(v) for v in times.tolist()]
+    ms_a, ms_b, ms_total = max_over_ranks([ms_a, ms_b, ms_total], dist, device)
 
     # ---------------- end to end through the public API with HOST buffers ----------------
     e2e = measure_e2e(P, layer, device, dist, steps=max(2, min(K, 5)))
@@ -242,8 +254,8 @@ def run_ours(args):
         return
     peaks, peak_kind = measured_peaks()
     qbytes, lops = quantizer_bytes(), linear_ops()
-    gbs = world * qbytes * K / (ms_a * 1e-3) / 1e9
-    tops = world * lops * K / (ms_b * 1e-3) / 1e12
+    gbs = throughput(world, qbytes, K, ms_a) / 1e9
+    tops = throughput(world, lops, K, ms_b) / 1e12
     int8_peak = peaks["bf16_tflops_sustained"] * INT8_OVER_BF16_NOMINAL
     ach_q = qbytes * K / (ms_a * 1e-3) / 1e9            # per GPU
     ach_l = lops * K / (ms_b * 1e-3) / 1e12
@@ -305,12 +317,8 @@ def measure_e2e(P, layer, device, dist, steps: int):
         step()
     e1.record(stream)
     torch.cuda.synchronize()
-    ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=device)
-    world = 1
-    if dist is not None:
-        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-        world = dist.get_world_size()
-    ms = float(ms.item()) / steps
+    world = 1 if dist is None else dist.get_world_size()
+    ms = max_over_ranks([e0.elapsed_time(e1)], dist, device)[0] / steps
     return {"value": round(world * quantizer_bytes() / (ms * 1e-3) / 1e9, 2), "unit": "GB/s",
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(ms, 4), "steps": steps,
             "w8a8_tops": round(world * linear_ops() / (ms * 1e-3) / 1e12, 3)}
@@ -347,8 +355,14 @@ def _oracle_sample(gemm_rows: int):
     return t_q, t_l, ops
 
 
-def cpu_baseline(gemm_rows: int = 128):
+def cpu_baseline(budget_seconds: float = 25.0):
     import oracle
+    # the whole step if the oracle can do it within the budget on this host, otherwise as many GEMM rows as fit
+    # (sized from a 64-row probe); the quantizer part always runs on the full tensors
+    _, t_probe, _ = _oracle_sample(64)
+    gemm_rows = T_TOKENS if t_probe * (T_TOKENS / 64) <= budget_seconds else \
+        int(max(64, 64 * budget_seconds / max(t_probe, 1e-3)))
+    gemm_rows -= gemm_rows % 8
     t_q, t_l, ops = _oracle_sample(gemm_rows)
     # the oracle runs forward and backward as two passes: 4 + 6 algorithmic bytes per element;
     # the reported GB/s uses the step's 8 bytes per element so that it is the same metric
