@@ -13,7 +13,8 @@ namespace {
 
 // launch shape of the streaming kernel
 constexpr int kThreads = 256;
-constexpr int kUnroll = 2;
+constexpr int kUnroll = 2;             // 128-bit vectors of x (and of g) in flight per thread
+constexpr int kUnrollFwdOnly = 4;      // the forward alone loads half as much per vector: keep as many bytes in flight
 constexpr int kBlocksPerSM = 4;
 constexpr int kLoadHint = 1;
 constexpr int kStoreHint = 1;
@@ -58,7 +59,7 @@ cudaError_t launch_stream(const QParams& p, int grid, cudaStream_t st) {
     cudaLaunchAttribute attr[1] = {pdl_attribute()};
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, fakequant_kernel<BF, FWD, BWD, kThreads, kUnroll, kBlocksPerSM, kLoadHint, kStoreHint>, p);
+    return cudaLaunchKernelEx(&cfg, fakequant_kernel<BF, FWD, BWD, kThreads, (BWD ? kUnroll : kUnrollFwdOnly), kBlocksPerSM, kLoadHint, kStoreHint>, p);
 }
 
 template <bool BF>

@@ -312,8 +312,9 @@ constexpr int P_STAGE_BYTES = P_A_BYTES + P_B_BYTES_MAX;
 
 constexpr int P_NUM_THREADS = 448;       // 14 warps: producer, MMA issuer, 4 epilogue, 8 activation quantizer
 constexpr int CONV_THREADS = 256;
-constexpr int CONV_ITEMS = 16;           // 8-element items per thread and chunk: 16 128-bit loads in flight per thread
-constexpr int CONV_CHUNK = CONV_THREADS * CONV_ITEMS;   // items per chunk (32768 elements)
+constexpr int CONV_WARPS = CONV_THREADS / 32;
+constexpr int CONV_ITEMS = 16;           // 8-element items per lane and chunk: 16 128-bit loads in flight per lane
+constexpr int CONV_CHUNK = 32 * CONV_ITEMS;   // items per chunk: one warp, 4096 elements
 constexpr int kMaxRowBlocks = 1024;      // 256-row blocks the in-kernel quantizer can publish (T <= 262144)
 constexpr int kReadySlots = 32;          // concurrently running launches that can each own a set of counters
 
@@ -393,6 +394,61 @@ __device__ __forceinline__ uint4 ld_stream16(const uint4* p) {
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;
+}
+
+// ---- in-kernel activation quantizer: one chunk = 32 lanes x CONV_ITEMS items of 8 elements, contiguous in x ----
+struct ConvJob {
+    const uint4* src;            // x as 128-bit words (8 elements each)
+    uint2* dst;                  // int8 codes as 64-bit words
+    unsigned* ready;             // per 256-row block: items quantized and visible
+    long long total;             // items in x
+    long long items_per_block;   // items per 256-row block
+    float inv, qn, qp;
+    bool eight;
+};
+
+__device__ __forceinline__ void conv_load(const ConvJob& j, long long c, int lane, uint4 (&v)[CONV_ITEMS]) {
+#pragma unroll
+    for (int u = 0; u < CONV_ITEMS; ++u) {
+        const long long i = c * CONV_CHUNK + u * 32 + lane;
+        if (i < j.total) v[u] = ld_stream16(j.src + i);
+    }
+}
+
+template <bool BF>
+__device__ __forceinline__ void conv_store(const ConvJob& j, long long c, int lane, const uint4 (&v)[CONV_ITEMS]) {
+    if (j.eight) {
+#pragma unroll
+        for (int u = 0; u < CONV_ITEMS; ++u) {
+            const long long i = c * CONV_CHUNK + u * 32 + lane;
+            if (i < j.total) j.dst[i] = quantize8<BF, true>(v[u], j.inv, j.qn, j.qp);
+        }
+    } else {
+#pragma unroll
+        for (int u = 0; u < CONV_ITEMS; ++u) {
+            const long long i = c * CONV_CHUNK + u * 32 + lane;
+            if (i < j.total) j.dst[i] = quantize8<BF, false>(v[u], j.inv, j.qn, j.qp);
+        }
+    }
+}
+
+// every lane's stores visible at GPU scope (and to the TMA unit), then one add per row block the chunk touches
+__device__ __forceinline__ void conv_publish(const ConvJob& j, long long c, int lane) {
+    asm volatile("fence.proxy.async.global;" ::: "memory");
+    __threadfence();
+    __syncwarp();
+    if (lane == 0) {
+        const long long first = c * CONV_CHUNK;
+        const long long end = (first + CONV_CHUNK < j.total) ? first + CONV_CHUNK : j.total;
+        long long i = first;
+        while (i < end) {
+            const long long blk = i / j.items_per_block;
+            const long long blk_end = (blk + 1) * j.items_per_block;
+            const long long upto = blk_end < end ? blk_end : end;
+            atomicAdd(j.ready + blk, (unsigned)(upto - i));
+            i = upto;
+        }
+    }
 }
 
 // Bounded wait until *counter (written by other CTAs with a fence before their atomic add) reaches `need`.
@@ -509,6 +565,22 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     const uint32_t tmem_base = tail->tmem_base;
     pdl_wait();                         // set-up done; from here on global memory of earlier kernels is used
 
+    // what the activation quantizer warps work on (and what the producers wait for)
+    ConvJob job{};
+    long long conv_chunks = 0;
+    if (pp.x != nullptr) {
+        job.src = reinterpret_cast<const uint4*>(pp.x);
+        job.dst = reinterpret_cast<uint2*>(pp.a_int8);
+        job.ready = pp.ready;
+        job.total = (long long)p.T * (p.K >> 3);
+        job.items_per_block = (long long)PBM * (p.K >> 3);
+        job.inv = __fdiv_rn(1.0f, __ldg(p.x_scale));
+        job.qn = pp.qn;
+        job.qp = pp.qp;
+        job.eight = pp.qp == 127.0f;
+        conv_chunks = (job.total + CONV_CHUNK - 1) / CONV_CHUNK;
+    }
+
     const int num_tiles = pp.pair_m_blocks * pp.n_tiles;
     const int pair_id = blockIdx.x >> 1;
     const int num_pairs = gridDim.x >> 1;
@@ -525,30 +597,44 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 int n0, bn;
                 pair_tile_cols(pp, tile - m_blk * pp.n_tiles, &n0, &bn);
                 const int a_row = m_blk * PBM + (int)rank * 128;
+                // this CTA's half of the tile's W rows; the box is as high as half the widest tile, so a narrower
+                // tile fetches 8 rows it does not use (rows past N read as zero)
+                const int w_row = n0 + (int)rank * (bn >> 1);
+                int kb_a = 0;            // k-blocks of this tile whose W half is already on its way
                 if (pp.x != nullptr && m_blk != ready_blk) {
-                    // the rows of this block must have been quantized, by whichever CTAs had them, and be visible
-                    // to the TMA unit before the first load of the tile
+                    // The rows of this block must have been quantized, by whichever CTAs had them, and be visible
+                    // to the TMA unit before the first A load of the tile.  W does not depend on that: while
+                    // waiting, fill the free stages with the W halves of the first k-blocks.
                     const int rows = p.T - m_blk * PBM;
-                    ok = wait_rows_ready(pp.ready + m_blk, (unsigned)((rows < PBM ? rows : PBM) * (p.K >> 3)), tail, p);
+                    const unsigned need = (unsigned)((rows < PBM ? rows : PBM) * (p.K >> 3));
+                    int st = stage;
+                    uint32_t ph = phase;
+                    while (kb_a < p.k_blocks && kb_a < P_STAGES && ptx::mbar_test_wait(&tail->empty[st], ph ^ 1u)) {
+                        const uint32_t full_leader = ptx::mapa_u32(ptx::smem_u32(&tail->full[st]), 0);
+                        if (rank == 0) ptx::mbar_arrive_expect_tx(&tail->full[st], 2u * stage_tx);
+                        ptx::tma_load_2d_pair(tiles + (size_t)st * P_STAGE_BYTES + P_A_BYTES, &tmap_w, full_leader,
+                                              kb_a * BK, w_row);
+                        ++kb_a;
+                        if (++st == P_STAGES) { st = 0; ph ^= 1u; }
+                    }
+                    ok = wait_rows_ready(pp.ready + m_blk, need, tail, p);
                     if (!ok) break;
                     asm volatile("fence.proxy.async.global;" ::: "memory");
                     ready_blk = m_blk;
                 }
-                // this CTA's half of the tile's W rows; the box is as high as half the widest tile, so a narrower
-                // tile fetches 8 rows it does not use (rows past N read as zero)
-                const int w_row = n0 + (int)rank * (bn >> 1);
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
-                    ok = wait_bounded_pair(&tail->empty[stage], phase ^ 1u, tail, p);
-                    if (!ok) break;
                     uint8_t* a_dst = tiles + (size_t)stage * P_STAGE_BYTES;
-                    uint8_t* b_dst = a_dst + P_A_BYTES;
                     // Only the leader arms the barrier (with the bytes of both CTAs); the partner's copies
                     // may complete first, which merely drives the transaction count negative for a while:
                     // the phase cannot complete before the leader's arrival.
                     const uint32_t full_leader = ptx::mapa_u32(ptx::smem_u32(&tail->full[stage]), 0);
-                    if (rank == 0) ptx::mbar_arrive_expect_tx(&tail->full[stage], 2u * stage_tx);
+                    if (kb >= kb_a) {
+                        ok = wait_bounded_pair(&tail->empty[stage], phase ^ 1u, tail, p);
+                        if (!ok) break;
+                        if (rank == 0) ptx::mbar_arrive_expect_tx(&tail->full[stage], 2u * stage_tx);
+                        ptx::tma_load_2d_pair(a_dst + P_A_BYTES, &tmap_w, full_leader, kb * BK, w_row);
+                    }
                     ptx::tma_load_2d_pair(a_dst, &tmap_a, full_leader, kb * BK, a_row);
-                    ptx::tma_load_2d_pair(b_dst, &tmap_w, full_leader, kb * BK, w_row);
                     if (++stage == P_STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -601,68 +687,19 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         __syncwarp();
     } else if (warp >= 6) {
         // ---------------- activation quantizer (warps 6..13 of both CTAs) ----------------
-        // x is taken as a flat run of T * K / 8 items of 8 elements, cut into chunks that are dealt round-robin
-        // over the CTAs in address order, so the row blocks become ready in the order the tiles need them.  Each
-        // thread keeps 16 128-bit loads in flight; the loads of a CTA's next chunk are issued before the fence and
-        // barrier that publish the current one, so their latencies overlap.
+        // x is taken as a flat run of T * K / 8 items of 8 elements, cut into chunks of 4096 elements that are
+        // dealt round-robin over all quantizer warps of the grid in address order, so the row blocks become ready
+        // in the order the tiles need them.  Every warp runs its own load -> quantize -> store -> fence -> publish
+        // pipeline with 16 128-bit loads in flight per lane; the warps drift apart, which keeps DRAM busy while
+        // some of them wait for their stores to be acknowledged.
         if (pp.x != nullptr) {
-            const int ct = threadIdx.x - (P_NUM_THREADS - CONV_THREADS);
-            const float inv = __fdiv_rn(1.0f, __ldg(p.x_scale));
-            const float qn = pp.qn, qp = pp.qp;
-            const bool eight = qp == 127.0f;
-            const long long items_per_block = (long long)PBM * (p.K >> 3);
-            const long long total = (long long)p.T * (p.K >> 3);
-            const long long n_chunks = (total + CONV_CHUNK - 1) / CONV_CHUNK;
-            const uint4* src = reinterpret_cast<const uint4*>(pp.x);
-            uint2* dst = reinterpret_cast<uint2*>(pp.a_int8);
-            uint4 v[CONV_ITEMS];
-            long long c = blockIdx.x;
-            if (c < n_chunks) {
-#pragma unroll
-                for (int u = 0; u < CONV_ITEMS; ++u) {
-                    const long long i = c * CONV_CHUNK + u * CONV_THREADS + ct;
-                    if (i < total) v[u] = ld_stream16(src + i);
-                }
-            }
-            while (c < n_chunks) {
-                if (eight) {
-#pragma unroll
-                    for (int u = 0; u < CONV_ITEMS; ++u) {
-                        const long long i = c * CONV_CHUNK + u * CONV_THREADS + ct;
-                        if (i < total) dst[i] = quantize8<BF, true>(v[u], inv, qn, qp);
-                    }
-                } else {
-#pragma unroll
-                    for (int u = 0; u < CONV_ITEMS; ++u) {
-                        const long long i = c * CONV_CHUNK + u * CONV_THREADS + ct;
-                        if (i < total) dst[i] = quantize8<BF, false>(v[u], inv, qn, qp);
-                    }
-                }
-                const long long cn = c + gridDim.x;
-                if (cn < n_chunks) {
-#pragma unroll
-                    for (int u = 0; u < CONV_ITEMS; ++u) {
-                        const long long i = cn * CONV_CHUNK + u * CONV_THREADS + ct;
-                        if (i < total) v[u] = ld_stream16(src + i);
-                    }
-                }
-                asm volatile("fence.proxy.async.global;" ::: "memory");
-                __threadfence();
-                asm volatile("bar.sync 3, 256;" ::: "memory");
-                if (ct == 0) {
-                    // credit the chunk's items to the row block(s) they lie in
-                    const long long first = c * CONV_CHUNK;
-                    const long long end = (first + CONV_CHUNK < total) ? first + CONV_CHUNK : total;
-                    long long i = first;
-                    while (i < end) {
-                        const long long blk = i / items_per_block;
-                        const long long blk_end = (blk + 1) * items_per_block;
-                        const long long upto = blk_end < end ? blk_end : end;
-                        atomicAdd(pp.ready + blk, (unsigned)(upto - i));
-                        i = upto;
-                    }
-                }
-                c = cn;
+            const int cw = warp - (P_NUM_THREADS - CONV_THREADS) / 32;          // 0..7
+            const long long stride = (long long)gridDim.x * CONV_WARPS;
+            for (long long c = (long long)blockIdx.x * CONV_WARPS + cw; c < conv_chunks; c += stride) {
+                uint4 v[CONV_ITEMS];
+                conv_load(job, c, lane, v);
+                conv_store<BF>(job, c, lane, v);
+                conv_publish(job, c, lane);
             }
         }
     } else {
