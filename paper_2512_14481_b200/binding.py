@@ -27,8 +27,9 @@ SASQ_BF16 = 1
 
 def linear_launches(T: int) -> int:
     """Kernels one sasq_static_w8a8_linear call launches, for launch counting: one when the activation quantizer
-    runs inside the GEMM kernel (128 < T <= 262144), otherwise the quantizer and the GEMM."""
-    return 1 if 128 < int(T) <= 262144 else 2
+    runs inside the GEMM kernel (T <= 262144 and, for T <= 128, at most one 128-channel tile per SM), otherwise
+    the quantizer and the GEMM."""
+    return 1 if int(T) <= 262144 else 2
 
 
 _HERE = os.path.dirname(os.path.abspath(__file__))

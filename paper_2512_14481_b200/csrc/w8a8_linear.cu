@@ -490,32 +490,6 @@ __device__ __forceinline__ bool wait_bounded_pair(uint64_t* bar, uint32_t parity
     return true;
 }
 
-template <bool BF, int NCOLS>
-__device__ __forceinline__ void epilogue_chunk(const uint32_t* v, const float* scale, const float* bias, bool has_bias,
-                                               bool row_ok, int n_base, int N, uint16_t* yrow, int32_t* arow) {
-#pragma unroll
-    for (int j = 0; j < NCOLS; j += 8) {
-        if (row_ok && (n_base + j) < N) {
-            uint32_t o[4];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                float f0 = __fmul_rn(__int2float_rn((int)v[j + 2 * q]), scale[j + 2 * q]);
-                float f1 = __fmul_rn(__int2float_rn((int)v[j + 2 * q + 1]), scale[j + 2 * q + 1]);
-                if (has_bias) {
-                    f0 = __fadd_rn(f0, bias[j + 2 * q]);
-                    f1 = __fadd_rn(f1, bias[j + 2 * q + 1]);
-                }
-                o[q] = narrow2<BF>(f0, f1);
-            }
-            *reinterpret_cast<uint4*>(yrow + j) = make_uint4(o[0], o[1], o[2], o[3]);
-            if (arow != nullptr) {
-                *reinterpret_cast<uint4*>(arow + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                *reinterpret_cast<uint4*>(arow + j + 4) = make_uint4(v[j + 4], v[j + 5], v[j + 6], v[j + 7]);
-            }
-        }
-    }
-}
-
 template <bool BF>
 __global__ void __launch_bounds__(P_NUM_THREADS, 1)
 w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
@@ -857,6 +831,305 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
 
 // Eq. 1 with the fixed factor, written once to int8 (operand A of the GEMM).
 // 16 elements per thread: two 128-bit loads, one 128-bit store.
+// ---------------------------------------------------------------------------
+// Small-T kernel (T <= 128: decode and short prompts).  The work is streaming W once from HBM, so the roles of the
+// operands are swapped: 128 rows of W are the M side of the MMA (every instruction consumes 4 KB of weights), the
+// T activation rows, padded to a multiple of 16, are the N side, and the accumulator tile in TMEM is
+// [128 output channels x T tokens].  To occupy the whole chip a cluster of S CTAs shares one 128-channel tile and
+// splits K; each CTA parks its partial accumulators in its own shared memory, and after a cluster barrier CTA r
+// adds the S partials of its 128 / S channels through distributed shared memory (int32: exact in any order),
+// dequantises and stores them.
+//   warp 0      TMA producer: W tile (128 x 128 B) + int8 activation tile (TP x 128 B) per stage
+//   warp 1      MMA issuer
+//   warps 2..5  first the activation quantizer (Eq. 1 with the fixed factor, all CTAs share the T x K elements and
+//               publish through one counter; the producers load activation tiles only after it is complete, the
+//               weight tiles of the first stages are on their way by then), then the epilogue
+// ---------------------------------------------------------------------------
+constexpr int D_THREADS = 192;
+constexpr int D_W_BYTES = 128 * BK;          // weight tile of a stage
+constexpr int D_MAX_STAGES = 8;
+constexpr int D_RING_BYTES = 192 * 1024;     // stages x (weight tile + activation tile) fit in here
+
+struct DecodeTail {
+    uint64_t full[D_MAX_STAGES];
+    uint64_t empty[D_MAX_STAGES];
+    uint64_t acc_full;
+    uint32_t tmem_base;
+    volatile int abort_flag;
+    int is_last_cta;
+};
+
+struct DecodeParams {
+    LinearParams lp;
+    int tp;              // T rounded up to a multiple of 16: N of the MMA
+    int stages;
+    int split;           // CTAs per cluster = K slices
+    int n_tiles;         // 128-channel tiles
+    uint32_t tmem_cols;  // power of two >= max(32, tp)
+    const uint16_t* x;
+    uint8_t* a_int8;
+    unsigned* ready;     // [1] 16-element items quantized and visible; zero at launch
+    unsigned* done;
+    float qn, qp;
+};
+
+__device__ __forceinline__ bool wait_bounded_d(uint64_t* bar, uint32_t parity, DecodeTail* tail, const LinearParams& p) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    int polls = 0;
+    while (!ptx::mbar_try_wait(bar, parity)) {
+        if ((++polls & 63) == 0) {
+            if (tail->abort_flag) return false;
+            if (clock64() - t0 > p.wait_limit) {
+                tail->abort_flag = 1;
+                atomicMax(p.status, (int)SASQ_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+template <bool BF>
+__global__ void __launch_bounds__(D_THREADS, 1)
+w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
+                   const __grid_constant__ DecodeParams dp) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t* ring = smem_raw;
+    DecodeTail* tail = reinterpret_cast<DecodeTail*>(ring + D_RING_BYTES);
+    const LinearParams& p = dp.lp;
+    if ((ptx::smem_u32(ring) & 1023u) != 0) {       // uniform over the grid: every CTA returns before any barrier
+        if (threadIdx.x == 0) atomicMax(p.status, (int)SASQ_ERR_CUDA);
+        return;
+    }
+    pdl_launch_dependents();
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int rank = (int)ptx::cluster_ctarank();
+    const int n_tile = blockIdx.x / dp.split;
+    const int n0 = n_tile * 128;
+    const int stage_bytes = D_W_BYTES + dp.tp * BK;
+    // this CTA's slice of the k-blocks
+    const int kb_begin = (int)(((long long)rank * p.k_blocks) / dp.split);
+    const int kb_end = (int)(((long long)(rank + 1) * p.k_blocks) / dp.split);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < dp.stages; ++s) {
+            ptx::mbar_init(&tail->full[s], 1);
+            ptx::mbar_init(&tail->empty[s], 1);
+        }
+        ptx::mbar_init(&tail->acc_full, 1);
+        tail->abort_flag = 0;
+        ptx::mbar_init_fence();
+        ptx::prefetch_tensormap(&tmap_w);
+        ptx::prefetch_tensormap(&tmap_x);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(&tail->tmem_base, dp.tmem_cols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = tail->tmem_base;
+    pdl_wait();                         // set-up done; from here on global memory of earlier kernels is used
+
+    const unsigned items_total = (unsigned)(((long long)p.T * p.K) >> 4);      // 16 elements each
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (ptx::elect_one()) {
+            bool ok = true;
+            int stage = 0;
+            uint32_t phase = 0;
+            // weight tiles of the first stages go out at once; the activation tiles follow when every CTA has
+            // quantized its share of x
+            int early = kb_end - kb_begin < dp.stages ? kb_end - kb_begin : dp.stages;
+            for (int i = 0; i < early; ++i) {
+                ptx::mbar_arrive_expect_tx(&tail->full[i], (uint32_t)stage_bytes);
+                ptx::tma_load_2d(ring + (size_t)i * stage_bytes, &tmap_w, &tail->full[i], (kb_begin + i) * BK, n0);
+            }
+            {
+                const long long t0 = clock64();
+                int polls = 0;
+                for (;;) {
+                    unsigned v;
+                    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(dp.ready) : "memory");
+                    if (v >= items_total) break;
+                    if ((++polls & 15) == 0) {
+                        if (tail->abort_flag) { ok = false; break; }
+                        if (clock64() - t0 > p.wait_limit) {
+                            tail->abort_flag = 1;
+                            atomicMax(p.status, (int)SASQ_ERR_TIMEOUT);
+                            ok = false;
+                            break;
+                        }
+                    }
+                    __nanosleep(32);
+                }
+                asm volatile("fence.proxy.async.global;" ::: "memory");
+            }
+            for (int kb = kb_begin; kb < kb_end && ok; ++kb) {
+                uint8_t* w_dst = ring + (size_t)stage * stage_bytes;
+                if (kb - kb_begin >= early) {
+                    ok = wait_bounded_d(&tail->empty[stage], phase ^ 1u, tail, p);
+                    if (!ok) break;
+                    ptx::mbar_arrive_expect_tx(&tail->full[stage], (uint32_t)stage_bytes);
+                    ptx::tma_load_2d(w_dst, &tmap_w, &tail->full[stage], kb * BK, n0);
+                }
+                ptx::tma_load_2d(w_dst + D_W_BYTES, &tmap_x, &tail->full[stage], kb * BK, 0);
+                if (++stage == dp.stages) { stage = 0; phase ^= 1u; }
+            }
+            if (!ok) {      // copies in flight must land before the CTA's shared memory goes away
+                const long long t0 = clock64();
+                while (clock64() - t0 < (1LL << 22)) __nanosleep(1000);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (ptx::elect_one()) {
+            const uint32_t idesc = ptx::idesc_i8(128, dp.tp);
+            const uint64_t w_desc0 = ptx::smem_desc_k_major_sw128(ptx::smem_u32(ring));
+            const uint64_t x_desc0 = ptx::smem_desc_k_major_sw128(ptx::smem_u32(ring) + D_W_BYTES);
+            const uint32_t stage_step = (uint32_t)(stage_bytes >> 4);
+            int stage = 0;
+            uint32_t phase = 0;
+            uint32_t accumulate = 0;
+            bool ok = true;
+            for (int kb = kb_begin; kb < kb_end; ++kb) {
+                ok = wait_bounded_d(&tail->full[stage], phase, tail, p);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                const uint64_t w_desc = w_desc0 + (uint64_t)(stage * stage_step);
+                const uint64_t x_desc = x_desc0 + (uint64_t)(stage * stage_step);
+                ptx::mma_i8_ss(tmem_base, w_desc, x_desc, idesc, accumulate);
+                ptx::mma_i8_ss_acc(tmem_base, w_desc + 2, x_desc + 2, idesc);
+                ptx::mma_i8_ss_acc(tmem_base, w_desc + 4, x_desc + 4, idesc);
+                ptx::mma_i8_ss_acc(tmem_base, w_desc + 6, x_desc + 6, idesc);
+                accumulate = 1u;
+                ptx::mma_commit(&tail->empty[stage]);
+                if (++stage == dp.stages) { stage = 0; phase ^= 1u; }
+            }
+            if (ok) ptx::mma_commit(&tail->acc_full);       // also right for an empty slice: arrives at once
+        }
+        __syncwarp();
+    } else {
+        // ---------------- activation quantizer, then epilogue (warps 2..5) ----------------
+        const int et = threadIdx.x - 64;                       // 0..127
+        const float sx = __ldg(p.x_scale);
+        if (blockIdx.x == 0 && et == 0 && scale_is_bad(sx)) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
+        {
+            const float inv = __fdiv_rn(1.0f, sx);
+            const uint4* src = reinterpret_cast<const uint4*>(dp.x);
+            uint4* dst = reinterpret_cast<uint4*>(dp.a_int8);
+            unsigned mine = 0;
+            for (unsigned i = blockIdx.x * 128u + (unsigned)et; i < items_total; i += gridDim.x * 128u) {
+                const uint4 a = ld_stream16(src + 2 * (size_t)i), b = ld_stream16(src + 2 * (size_t)i + 1);
+                const uint2 lo = quantize8<BF, false>(a, inv, dp.qn, dp.qp);
+                const uint2 hi = quantize8<BF, false>(b, inv, dp.qn, dp.qp);
+                dst[i] = make_uint4(lo.x, lo.y, hi.x, hi.y);
+                ++mine;
+            }
+            asm volatile("fence.proxy.async.global;" ::: "memory");
+            __threadfence();
+            // one add per warp
+            for (int off = 16; off > 0; off >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, off);
+            if (lane == 0 && mine != 0) atomicAdd(dp.ready, mine);
+        }
+
+        // epilogue part 1: this CTA's partial accumulators, TMEM -> own shared memory (over the drained ring),
+        // rows = channels, tp + 4 words apart: 128-bit accesses stay aligned and eight consecutive rows cover
+        // all banks, so neither these stores nor the reads below conflict
+        const int quad = warp & 3;                              // TMEM lane quadrant of this warp
+        const int pstride = dp.tp + 4;
+        int32_t* part = reinterpret_cast<int32_t*>(ring);
+        bool ok = wait_bounded_d(&tail->acc_full, 0u, tail, p);
+        ok = epilogue_all_ok(ok);
+        if (ok) {
+            ptx::tc_fence_after_sync();
+            uint4* prow = reinterpret_cast<uint4*>(part + (size_t)(quad * 32 + lane) * pstride);
+            if (kb_end > kb_begin) {
+                const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
+                for (int c = 0; c < dp.tp; c += 16) {
+                    uint32_t v[16];
+                    ptx::tmem_ld_32x16(taddr + (uint32_t)c, v);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        prow[(c >> 2) + j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                }
+            } else {
+                for (int c = 0; c < dp.tp; c += 4) prow[c >> 2] = make_uint4(0u, 0u, 0u, 0u);
+            }
+        }
+        ptx::tc_fence_before_sync();
+    }
+
+    // every CTA's partials are in place (or the launch has been abandoned: a role gave up after a bounded wait and
+    // the status word says so; the sums below are then garbage but every access stays in bounds)
+    __syncthreads();
+    ptx::cluster_sync_all();
+
+    if (warp >= 2) {
+        // epilogue part 2: CTA r reduces channels [r * 128 / S, (r + 1) * 128 / S) of the tile over the S partials.
+        // One work item = one channel x four consecutive tokens (one 128-bit read per partial); consecutive
+        // threads take consecutive channels so that the 16-bit stores of one token coalesce.
+        const int et = threadIdx.x - 64;
+        const int rows = 128 / dp.split;
+        const int pstride = dp.tp + 4;
+        const bool has_bias = p.bias != nullptr;
+        const float sx = __ldg(p.x_scale);
+        const int items = rows * (dp.tp >> 2);
+        for (int it = et; it < items; it += 128) {
+            const int n_local = rank * rows + (it % rows);
+            const int t0 = (it / rows) << 2;
+            const int n = n0 + n_local;
+            const uint32_t my = ptx::smem_u32(ring) + (uint32_t)(n_local * pstride + t0) * 4u;
+            int32_t acc[4] = {0, 0, 0, 0};
+            for (int r = 0; r < dp.split; ++r) {
+                int32_t v0, v1, v2, v3;
+                const uint32_t addr = ptx::mapa_u32(my, (uint32_t)r);
+                asm volatile("ld.shared::cluster.v4.s32 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3) : "r"(addr) : "memory");
+                acc[0] += v0; acc[1] += v1; acc[2] += v2; acc[3] += v3;
+            }
+            if (n < p.N) {
+                const float sc = __fmul_rn(sx, __ldg(p.w_scale + n));
+                const float bv = has_bias ? widen1<BF>(__ldg(reinterpret_cast<const uint16_t*>(p.bias) + n)) : 0.0f;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int t = t0 + j;
+                    if (t < p.T) {
+                        float f = __fmul_rn(__int2float_rn(acc[j]), sc);
+                        if (has_bias) f = __fadd_rn(f, bv);
+                        reinterpret_cast<uint16_t*>(p.y)[(size_t)t * p.N + n] = narrow1<BF>(f);
+                        if (p.acc_out != nullptr) p.acc_out[(size_t)t * p.N + n] = acc[j];
+                    }
+                }
+            }
+        }
+    }
+
+    // ---------------- teardown ----------------
+    // no CTA may leave while a peer can still read its partials
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::cluster_sync_all();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, dp.tmem_cols);
+    }
+    // the CTA that finishes last leaves the counters at zero for the next launch that draws them
+    if (threadIdx.x == 0) {
+        if (atomicAdd(dp.done, 1u) == gridDim.x - 1) {
+            *dp.ready = 0u;
+            *dp.done = 0u;
+        }
+    }
+}
+
 // The same quantizer as a launch of its own (small T, or more row blocks than the in-kernel counters hold):
 // 8 elements per thread and step, one 128-bit load, one 64-bit store.
 template <bool BF>
@@ -1003,6 +1276,44 @@ int pair_capacity(bool bf, int sm_count) {
     return clusters;
 }
 
+// Largest K split (CTAs per cluster) of the small-T kernel with which all n_tiles clusters are resident at once (the
+// in-kernel activation quantizer needs every CTA of the grid running); 0 if even one CTA per tile does not fit.
+int decode_split(bool bf, int n_tiles, int k_blocks, int sm_count, size_t smem_bytes) {
+    static int ready[64][2] = {};
+    static int cap[64][2][4] = {};            // resident clusters for S = 1, 2, 4, 8; 0 = not asked yet
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    const void* fn = bf ? reinterpret_cast<const void*>(w8a8_decode_kernel<true>)
+                        : reinterpret_cast<const void*>(w8a8_decode_kernel<false>);
+    if (!ready[dev][bf]) {
+        if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
+            return 0;
+        ready[dev][bf] = 1;
+    }
+    for (int si = 3; si >= 0; --si) {
+        const int S = 1 << si;
+        if (S > k_blocks || (long long)n_tiles * S > sm_count) continue;
+        if (cap[dev][bf][si] == 0) {
+            cudaLaunchConfig_t cfg{};
+            cfg.gridDim = dim3((unsigned)(sm_count / S * S), 1, 1);
+            cfg.blockDim = dim3(D_THREADS, 1, 1);
+            cfg.dynamicSmemBytes = smem_bytes;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = (unsigned)S;
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            int clusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&clusters, fn, &cfg) != cudaSuccess || clusters <= 0) clusters = -1;
+            cap[dev][bf][si] = clusters;
+        }
+        if (cap[dev][bf][si] >= n_tiles) return S;
+    }
+    return 0;
+}
+
 // Column tiling of a 256-row block for `pairs` resident CTA pairs.  One MMA of N columns keeps the tensor pipe
 // busy for about max(N, 208) / 2 cycles (below 208 columns the instruction is bound by reading its A operand), and a
 // launch takes as long as its fullest pair: waves x that cost of the widest tile.  Tiles are at least 16 x 8 = 128
@@ -1111,7 +1422,12 @@ int sasq_static_w8a8_linear(const void* x, const int8_t* w, const float* w_scale
     //    used and the row blocks fit its counters, otherwise by a launch of its own
     uint8_t* a_int8 = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(workspace) + 127) & ~uintptr_t(127));
     const float qn = (float)(1 << (bits - 1)), qp = (float)((1 << (bits - 1)) - 1);
-    const bool in_kernel_quantizer = T > BM && (T + PBM - 1) / PBM <= kMaxRowBlocks;
+    const int k_blocks = (int)((K + BK - 1) / BK);
+    constexpr size_t kDecodeSmem = (size_t)D_RING_BYTES + sizeof(DecodeTail);
+    const int n_tiles128 = (int)((N + 127) / 128);
+    const int split = (T <= BM && n_tiles128 <= sm_count)
+                          ? decode_split(dt == SASQ_BF16, n_tiles128, k_blocks, sm_count, kDecodeSmem) : 0;
+    const bool in_kernel_quantizer = split > 0 || (T > BM && (T + PBM - 1) / PBM <= kMaxRowBlocks);
     if (!in_kernel_quantizer) {
         const long long n8 = (T * K) / 8;     // K % 16 == 0
         long long blocks = (n8 + 255) / 256;
@@ -1135,12 +1451,47 @@ int sasq_static_w8a8_linear(const void* x, const int8_t* w, const float* w_scale
     p.y = y;
     p.acc_out = acc_out;
     p.T = (int)T; p.N = (int)N; p.K = (int)K;
-    p.k_blocks = (int)((K + BK - 1) / BK);
+    p.k_blocks = k_blocks;
     p.status = status;
     p.wait_limit = kWaitLimit;
     CUtensorMap tmap_a, tmap_w;
     cudaError_t e;
-    if (T > BM) {
+    if (split > 0) {
+        // small T: 128-channel tiles, K split over a cluster, activations quantized inside the kernel
+        DecodeParams dp{};
+        p.m_blocks = 1;
+        p.n_blocks = n_tiles128;
+        dp.lp = p;
+        dp.tp = (int)((T + 15) / 16) * 16;
+        const int stage_bytes = D_W_BYTES + dp.tp * BK;
+        dp.stages = D_RING_BYTES / stage_bytes < D_MAX_STAGES ? D_RING_BYTES / stage_bytes : D_MAX_STAGES;
+        dp.split = split;
+        dp.n_tiles = n_tiles128;
+        dp.tmem_cols = 32;
+        while ((int)dp.tmem_cols < dp.tp) dp.tmem_cols <<= 1;
+        dp.x = static_cast<const uint16_t*>(x);
+        dp.a_int8 = a_int8;
+        dp.qn = qn;
+        dp.qp = qp;
+        if (!next_ready_slot(&dp.ready, &dp.done)) return SASQ_ERR_CUDA;
+        if (!make_tmap(&tmap_w, w, N, K, 128) || !make_tmap(&tmap_a, a_int8, T, K, dp.tp)) return SASQ_ERR_CUDA;
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((unsigned)(n_tiles128 * split), 1, 1);
+        cfg.blockDim = dim3(D_THREADS, 1, 1);
+        cfg.dynamicSmemBytes = kDecodeSmem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)split;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        attr[1] = pdl_attribute();
+        cfg.attrs = attr;
+        cfg.numAttrs = 2;
+        if (dt == SASQ_BF16) e = cudaLaunchKernelEx(&cfg, w8a8_decode_kernel<true>, tmap_w, tmap_a, dp);
+        else e = cudaLaunchKernelEx(&cfg, w8a8_decode_kernel<false>, tmap_w, tmap_a, dp);
+        if (e != cudaSuccess) return SASQ_ERR_CUDA;
+    } else if (T > BM) {
         // CTA pairs, 256-row blocks cut into evenly wide column tiles that fill whole waves of the resident pairs
         const int pairs = pair_capacity(dt == SASQ_BF16, sm_count);
         if (pairs <= 0) return SASQ_ERR_CUDA;
