@@ -266,7 +266,8 @@ def run_ours(args):
         "data": "synthetic",
         "config": {"workload": WORKLOAD, "tokens": T_TOKENS, "bits": BITS, "tensors": 7,
                    "phases": "A: fused fake-quant fwd+bwd + scale-gradient reduction; B: 7 static W8A8 linears",
-                   "l2": "inputs larger than L2 (583 MB streamed in phase A, 348 MB of weights+activations in phase B)",
+                   "l2": f"inputs larger than L2 ({qbytes / 1e6:.0f} MB streamed in phase A, "
+                         f"{(202.4e6 + 2 * qbytes / 8) / 1e6:.0f} MB of weights+activations in phase B)",
                    "parallelism": "replicas" if world > 1 else "single"},
         "ms_phase_a": round(ms_a / K, 5), "ms_phase_b": round(ms_b / K, 5),
         "w8a8_linear": {"value": round(tops, 2), "unit": "TOPS", "ops_per_step": lops,
@@ -359,10 +360,11 @@ def cpu_baseline(budget_seconds: float = 25.0):
     import oracle
     # the whole step if the oracle can do it within the budget on this host, otherwise as many GEMM rows as fit
     # (sized from a 64-row probe); the quantizer part always runs on the full tensors
-    _, t_probe, _ = _oracle_sample(64)
-    gemm_rows = T_TOKENS if t_probe * (T_TOKENS / 64) <= budget_seconds else \
+    _, t_probe, _ = _oracle_sample(min(64, T_TOKENS))
+    gemm_rows = T_TOKENS if t_probe * max(1.0, T_TOKENS / 64) <= budget_seconds else \
         int(max(64, 64 * budget_seconds / max(t_probe, 1e-3)))
-    gemm_rows -= gemm_rows % 8
+    if gemm_rows >= 8:
+        gemm_rows -= gemm_rows % 8
     t_q, t_l, ops = _oracle_sample(gemm_rows)
     # the oracle runs forward and backward as two passes: 4 + 6 algorithmic bytes per element;
     # the reported GB/s uses the step's 8 bytes per element so that it is the same metric
@@ -380,7 +382,7 @@ def run_reference(args):
         return
     import oracle
     K = max(1, args.steps)
-    rows = 32
+    rows = min(32, T_TOKENS)
     for _ in range(min(args.warmup, 1)):
         _oracle_sample(rows)
     t_q = t_l = 0.0
@@ -418,7 +420,16 @@ def main():
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--tokens", type=int, default=2048,
+                    help="tokens per step (default 2048, the headline workload; other values time the same layer at "
+                         "decode or longer-prefill sizes and are named as such in config.workload)")
     args = ap.parse_args()
+    global T_TOKENS, WORKLOAD
+    if args.tokens != T_TOKENS:
+        if args.tokens < 1:
+            ap.error("--tokens must be positive")
+        T_TOKENS = args.tokens
+        WORKLOAD = f"llama2_7b_decoder_layer_7_linear_inputs_T{T_TOKENS}_bf16"
     if args.impl == "reference":
         run_reference(args)
     else:
