@@ -43,6 +43,10 @@ BITS = 8
 CONFIG_ID = 2
 L2_BYTES = 126 * 1024 * 1024
 INT8_OVER_BF16_NOMINAL = 2.0          # dense INT8 peak is twice the dense bf16 peak (4.5 vs 2.25 P-op/s nominal)
+# DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/ (T = 2048 workload only;
+# set to None whenever the kernel changes after its capture)
+NCU_TRAFFIC_FAKEQUANT = 532.5e6        # profiles/fakequant_kernel_llama7b_layer_T2048.md
+NCU_TRAFFIC_GEMM_MEAN = 467.9e6 / 7    # profiles/w8a8_gemm_pair_kernel_T2048.md: mean over the step's seven launches
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -272,13 +276,16 @@ def run_ours(args):
         "ms_phase_a": round(ms_a / K, 5), "ms_phase_b": round(ms_b / K, 5),
         "w8a8_linear": {"value": round(tops, 2), "unit": "TOPS", "ops_per_step": lops,
                         "frac_of_nominal_int8_4500": round(tops / world / 4500.0, 4)},
-        "roofline": {"kernel": "w8a8_gemm_kernel (tcgen05 int8)", "bound": "tensor", "achieved": round(ach_l, 2),
+        "roofline": {"kernel": "w8a8_gemm_pair_kernel (tcgen05 int8, CTA pairs, activation quantizer inside)",
+                     "bound": "tensor", "achieved": round(ach_l, 2),
                      "peak": round(int8_peak, 1), "unit": "TOP/s", "frac": round(ach_l / int8_peak, 4),
-                     "traffic": None,
+                     "traffic": (NCU_TRAFFIC_GEMM_MEAN if T_TOKENS == 2048 else None),
+                     "traffic_note": "DRAM bytes per launch, mean over the step's seven launches",
                      "peak_source": f"{peak_kind} sustained bf16 cuBLAS x 2 (nominal int8:bf16 ratio)"},
         "roofline_quantizer": {"kernel": "fakequant_kernel (fused fwd+bwd)", "bound": "hbm", "achieved": round(ach_q, 1),
                                "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(ach_q / peaks["hbm_gbs"], 4),
-                               "frac_of_nominal_8000": round(ach_q / 8000.0, 4), "traffic": None,
+                               "frac_of_nominal_8000": round(ach_q / 8000.0, 4),
+                               "traffic": (NCU_TRAFFIC_FAKEQUANT if T_TOKENS == 2048 else None),
                                "peak_source": f"{peak_kind} copy bandwidth"},
         "e2e": e2e, "gpu_launches": launches, "clocks": clocks, "wall_s": round(t_wall, 3),
     }
