@@ -149,6 +149,26 @@ SASQ_API int sasq_fakequant_fwd_bwd_multi(const sasq_qdesc_t* descs_host, int n_
                                  float* grad_scales_dev, int n_scales, int accumulate, int dt, int bits,
                                  void* workspace, size_t ws_bytes, void* stream);
 
+/* Bytes of scratch the per-channel call needs when it has a backward part. */
+SASQ_API size_t sasq_fakequant_per_channel_workspace(int64_t T, int64_t K);
+
+/* The fake-quant operator with one factor per channel (per column of x[T, K]), the granularity of the paper's
+ * experiments (Fig. 2b; Sec. 5.1: activations and weights both per channel).  Per element the arithmetic is that
+ * of the per-tensor calls with s = scales[k]; the gradient of factor k is summed over the T rows of column k:
+ *   y[t,k]  = narrow( fl32(c * scales[k]) ),   grad_x[t,k] = m ? grad_y[t,k] : +0,
+ *   grad_scales[k] = sum_t grad_y[t,k] * (m ? (r - t') : c)       (t' = fl32(x * fl32(1/scales[k])))
+ * x, y, grad_y, grad_x: [T, K] of `dt`; y == NULL skips the forward output, grad_y == grad_x == NULL skips the
+ * backward; y may alias x and grad_x may alias grad_y.  scales_dev, grad_scales_dev: [K] fp32, 16-byte aligned;
+ * grad_scales_dev is overwritten (accumulate == 0) or added to.  The sum runs in double per thread down the rows
+ * of a row group, then over the row groups in a fixed order: bit-identical from run to run, within 1e-4 relative
+ * of a double-precision sum.  workspace: >= sasq_fakequant_per_channel_workspace(T, K) bytes when there is a
+ * backward part.  K % 8 == 0, otherwise SASQ_ERR_UNSUPPORTED.  Any zero / non-finite factor sets
+ * SASQ_ERR_BAD_SCALE in the status word. */
+SASQ_API int sasq_fakequant_fwd_bwd_per_channel(const void* x, const void* grad_y, void* y, void* grad_x,
+                                                float* grad_scales_dev, int accumulate, int64_t T, int64_t K, int dt,
+                                                const float* scales_dev, int bits, void* workspace, size_t ws_bytes,
+                                                void* stream);
+
 /* Bytes of scratch sasq_static_w8a8_linear needs for this shape (may be 0). */
 SASQ_API size_t sasq_static_w8a8_linear_workspace(int64_t T, int64_t N, int64_t K);
 

@@ -19,6 +19,7 @@ __all__ = [
     "sasq_fakequant_multi_workspace", "sasq_fakequant_fwd_bwd_multi", "sasq_static_w8a8_linear_workspace",
     "sasq_static_w8a8_linear", "sasq_device_status", "QDesc", "sasq_absmax_scale_workspace", "sasq_absmax_scale",
     "sasq_quantize_weight", "linear_launches", "sasq_fakequant_fwd_bwd_static", "sasq_static_w8a8_linear_tiles",
+    "sasq_fakequant_per_channel_workspace", "sasq_fakequant_fwd_bwd_per_channel",
 ]
 
 SASQ_F16 = 0
@@ -84,6 +85,10 @@ def load_library() -> ctypes.CDLL:
     L.sasq_static_w8a8_linear_workspace.argtypes = [i64, i64, i64]
     L.sasq_static_w8a8_linear.restype = i32
     L.sasq_static_w8a8_linear.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, sz, vp]
+    L.sasq_fakequant_per_channel_workspace.restype = sz
+    L.sasq_fakequant_per_channel_workspace.argtypes = [i64, i64]
+    L.sasq_fakequant_fwd_bwd_per_channel.restype = i32
+    L.sasq_fakequant_fwd_bwd_per_channel.argtypes = [vp, vp, vp, vp, vp, i32, i64, i64, i32, vp, i32, vp, sz, vp]
     L.sasq_static_w8a8_linear_tiles.restype = i32
     L.sasq_static_w8a8_linear_tiles.argtypes = [i64, i64, i32, i32, ctypes.POINTER(ctypes.c_int32), i32]
     L.sasq_device_status.restype = i32
@@ -212,6 +217,34 @@ def sasq_fakequant_fwd_bwd_multi(tensors, scales, grad_scales, workspace, bits: 
                                                        int(bool(accumulate)), SASQ_BF16 if dt is None else dt,
                                                        int(bits), _ptr(workspace), _nbytes(workspace),
                                                        _stream(stream)), "sasq_fakequant_fwd_bwd_multi")
+
+
+def sasq_fakequant_per_channel_workspace(T: int, K: int) -> int:
+    return int(load_library().sasq_fakequant_per_channel_workspace(int(T), int(K)))
+
+
+def sasq_fakequant_fwd_bwd_per_channel(x, grad_y, y, grad_x, grad_scales, scales, workspace, bits: int = 8,
+                                       accumulate: bool = False, stream=None) -> None:
+    """x [T, K] with one factor per column: scales [K], grad_scales [K]; y or (grad_y, grad_x) may be None."""
+    _dev(x, "x"); _dev(scales, "scales", torch.float32)
+    if x.dim() != 2 or scales.numel() != x.shape[1]:
+        raise ValueError("x must be [T, K] and scales [K]")
+    for name, t in (("grad_y", grad_y), ("y", y), ("grad_x", grad_x)):
+        if t is not None:
+            _dev(t, name, x.dtype)
+            if tuple(t.shape) != tuple(x.shape):
+                raise ValueError(f"{name} must have the shape of x")
+    if grad_scales is not None:
+        _dev(grad_scales, "grad_scales", torch.float32)
+        if grad_scales.numel() != x.shape[1]:
+            raise ValueError("grad_scales must be [K]")
+    if workspace is not None:
+        _dev(workspace, "workspace")
+    _check(load_library().sasq_fakequant_fwd_bwd_per_channel(_ptr(x), _ptr(grad_y), _ptr(y), _ptr(grad_x),
+                                                             _ptr(grad_scales), int(bool(accumulate)), x.shape[0],
+                                                             x.shape[1], _dt(x), _ptr(scales), int(bits),
+                                                             _ptr(workspace), _nbytes(workspace), _stream(stream)),
+           "sasq_fakequant_fwd_bwd_per_channel")
 
 
 def sasq_static_w8a8_linear_workspace(T: int, N: int, K: int) -> int:

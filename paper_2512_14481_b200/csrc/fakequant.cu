@@ -9,6 +9,19 @@ SASQ_DEFINE_STATUS_WORD(g_fakequant_status)
 
 int fakequant_status_read_and_clear(cudaStream_t st) { return g_fakequant_status_read_and_clear(st); }
 
+// device address of the fake-quant status word on the current device (shared with the per-channel kernels)
+int* per_channel_status_ptr() {
+    static int* cache[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (cache[dev] == nullptr) {
+        int* p = nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_fakequant_status) != cudaSuccess) return nullptr;
+        cache[dev] = p;
+    }
+    return cache[dev];
+}
+
 namespace {
 
 // launch shape of the streaming kernel
