@@ -62,6 +62,13 @@ typedef enum {
 
 typedef enum { SASQ_F16 = 0, SASQ_BF16 = 1 } sasq_dtype_t;
 
+/* The fake-quant operator and the two ablations of Table 3. */
+typedef enum {
+    SASQ_FULL_OPERATOR = 0,   /* quant, round, clamp, dequant (Sec. 4.2) */
+    SASQ_WITHOUT_ROUND = 1,   /* "w/o round": r = t, so y = clamp(x / s) * s and the factor gradient inside the range is 0 */
+    SASQ_WITHOUT_CLAMP = 2    /* "w/o clamp": c = r, every element passes the gradient, term = r - t */
+} sasq_variant_t;
+
 /* One tensor of a multi-tensor fake-quant launch (host struct).  y == NULL skips
  * the forward output; grad_y == grad_x == NULL skips the backward; at least one
  * part must be present and every descriptor of one call must have the same
@@ -110,6 +117,13 @@ SASQ_API int sasq_fakequant_bwd(const void* x, const void* grad_y, void* grad_x,
 SASQ_API int sasq_fakequant_fwd_bwd(const void* x, const void* grad_y, void* y, void* grad_x, float* grad_scale_dev,
                            int accumulate, int64_t numel, int dt, const float* scale_dev, int bits,
                            void* workspace, size_t ws_bytes, void* stream);
+
+/* The fused pass with one of the operator's steps removed (Table 3's ablations; SASQ_FULL_OPERATOR gives
+ * sasq_fakequant_fwd_bwd).  Same arguments and conventions otherwise. */
+SASQ_API int sasq_fakequant_fwd_bwd_ablation(const void* x, const void* grad_y, void* y, void* grad_x,
+                                             float* grad_scale_dev, int accumulate, int64_t numel, int dt,
+                                             const float* scale_dev, int bits, int variant, void* workspace,
+                                             size_t ws_bytes, void* stream);
 
 /* The same fused pass for callers that can neither allocate device memory nor
  * hand over a workspace: for instance a plugin hook of an inference runtime that
@@ -215,6 +229,16 @@ SASQ_API int sasq_absmax_scale(const void* x, int64_t numel, int dt, int bits, f
  * w: [N, K] fp32; w_int: [N, K] int8; w_scale: [N] fp32. */
 SASQ_API int sasq_quantize_weight(const float* w, int8_t* w_int, float* w_scale, int64_t N, int64_t K, int bits,
                                   void* stream);
+
+/* One AdamW step on n factors (the factors are the only trainable parameters, Sec. 4.2; AdamW, lr 2e-4, Sec. 5.1),
+ * consuming the gradients the backward calls wrote, all in device memory, fp32:
+ *   m = beta1 m + (1 - beta1) g;   v = beta2 v + (1 - beta2) g^2;
+ *   s = s - lr * ( (m / (1 - beta1^step)) / (sqrt(v / (1 - beta2^step)) + eps) + weight_decay * s )
+ * scales_dev, exp_avg_dev (m), exp_avg_sq_dev (v): [n] fp32, updated in place; grad_scales_dev: [n] fp32.
+ * step counts from 1.  No constraint is put on the updated factors (Sec. 4.2). */
+SASQ_API int sasq_adamw_scales(float* scales_dev, const float* grad_scales_dev, float* exp_avg_dev,
+                               float* exp_avg_sq_dev, int n, int step, float lr, float beta1, float beta2, float eps,
+                               float weight_decay, void* stream);
 
 /* Synchronises `stream`, returns the sticky device status word of the current
  * device (SASQ_OK, SASQ_ERR_BAD_SCALE or SASQ_ERR_TIMEOUT) and clears it. */

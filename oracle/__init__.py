@@ -260,3 +260,17 @@ def w8a8_linear_grouped(x: np.ndarray, tag: int, w_int: np.ndarray, w_scale: np.
     _chk(lib().oracle_w8a8_linear_grouped(_p(x), _p(w_int), _p(w_scale), _p(s_group), _i64(group), _p(b), _p(y),
                                           _p(y32), _i64(T), _i64(N), _i64(K), ctypes.c_int(tag), ctypes.c_int(bits)))
     return y, y32
+
+
+def adamw_step(s, g, m, v, step: int, lr: float = 2e-4, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
+               weight_decay: float = 0.01):
+    """One AdamW step on the factors (Sec. 5.1: AdamW, lr 2e-4; the factors are the only trainable parameters,
+    Sec. 4.2), written out in float64 with decoupled weight decay.  Returns the new (s, m, v); inputs untouched."""
+    s = np.asarray(s, np.float64)
+    g = np.asarray(g, np.float64)
+    m = beta1 * np.asarray(m, np.float64) + (1.0 - beta1) * g
+    v = beta2 * np.asarray(v, np.float64) + (1.0 - beta2) * g * g
+    m_hat = m / (1.0 - beta1 ** step)
+    v_hat = v / (1.0 - beta2 ** step)
+    s_new = s - lr * (m_hat / (np.sqrt(v_hat) + eps) + weight_decay * s)
+    return s_new, m, v

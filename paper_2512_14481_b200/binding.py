@@ -20,10 +20,15 @@ __all__ = [
     "sasq_static_w8a8_linear", "sasq_device_status", "QDesc", "sasq_absmax_scale_workspace", "sasq_absmax_scale",
     "sasq_quantize_weight", "linear_launches", "sasq_fakequant_fwd_bwd_static", "sasq_static_w8a8_linear_tiles",
     "sasq_fakequant_per_channel_workspace", "sasq_fakequant_fwd_bwd_per_channel",
+    "sasq_fakequant_fwd_bwd_ablation", "sasq_adamw_scales", "SASQ_FULL_OPERATOR", "SASQ_WITHOUT_ROUND",
+    "SASQ_WITHOUT_CLAMP",
 ]
 
 SASQ_F16 = 0
 SASQ_BF16 = 1
+SASQ_FULL_OPERATOR = 0
+SASQ_WITHOUT_ROUND = 1
+SASQ_WITHOUT_CLAMP = 2
 
 
 def linear_launches(T: int) -> int:
@@ -85,6 +90,11 @@ def load_library() -> ctypes.CDLL:
     L.sasq_static_w8a8_linear_workspace.argtypes = [i64, i64, i64]
     L.sasq_static_w8a8_linear.restype = i32
     L.sasq_static_w8a8_linear.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, sz, vp]
+    L.sasq_fakequant_fwd_bwd_ablation.restype = i32
+    L.sasq_fakequant_fwd_bwd_ablation.argtypes = [vp, vp, vp, vp, vp, i32, i64, i32, vp, i32, i32, vp, sz, vp]
+    f32 = ctypes.c_float
+    L.sasq_adamw_scales.restype = i32
+    L.sasq_adamw_scales.argtypes = [vp, vp, vp, vp, i32, i32, f32, f32, f32, f32, f32, vp]
     L.sasq_fakequant_per_channel_workspace.restype = sz
     L.sasq_fakequant_per_channel_workspace.argtypes = [i64, i64]
     L.sasq_fakequant_fwd_bwd_per_channel.restype = i32
@@ -217,6 +227,32 @@ def sasq_fakequant_fwd_bwd_multi(tensors, scales, grad_scales, workspace, bits: 
                                                        int(bool(accumulate)), SASQ_BF16 if dt is None else dt,
                                                        int(bits), _ptr(workspace), _nbytes(workspace),
                                                        _stream(stream)), "sasq_fakequant_fwd_bwd_multi")
+
+
+def sasq_fakequant_fwd_bwd_ablation(x, grad_y, y, grad_x, grad_scale, scale, workspace, variant: int, bits: int = 8,
+                                    accumulate: bool = False, stream=None) -> None:
+    """The fused pass with Table 3's "w/o round" / "w/o clamp" ablations (variant = SASQ_WITHOUT_*)."""
+    _dev(x, "x"); _dev(grad_y, "grad_y", x.dtype); _dev(y, "y", x.dtype); _dev(grad_x, "grad_x", x.dtype)
+    _dev(grad_scale, "grad_scale", torch.float32); _dev(scale, "scale", torch.float32); _dev(workspace, "workspace")
+    if grad_y.numel() != x.numel() or grad_x.numel() != x.numel() or y.numel() != x.numel():
+        raise ValueError("grad_y, y and grad_x must have as many elements as x")
+    _check(load_library().sasq_fakequant_fwd_bwd_ablation(_ptr(x), _ptr(grad_y), _ptr(y), _ptr(grad_x),
+                                                          _ptr(grad_scale), int(bool(accumulate)), x.numel(), _dt(x),
+                                                          _ptr(scale), int(bits), int(variant), _ptr(workspace),
+                                                          _nbytes(workspace), _stream(stream)),
+           "sasq_fakequant_fwd_bwd_ablation")
+
+
+def sasq_adamw_scales(scales, grad_scales, exp_avg, exp_avg_sq, step: int, lr: float = 2e-4, beta1: float = 0.9,
+                      beta2: float = 0.999, eps: float = 1e-8, weight_decay: float = 0.01, stream=None) -> None:
+    """One AdamW step on the factors, in place (scales, exp_avg, exp_avg_sq: fp32 CUDA tensors of one size)."""
+    for name, t in (("scales", scales), ("grad_scales", grad_scales), ("exp_avg", exp_avg), ("exp_avg_sq", exp_avg_sq)):
+        _dev(t, name, torch.float32)
+        if t.numel() != scales.numel():
+            raise ValueError(f"{name} must have as many elements as scales")
+    _check(load_library().sasq_adamw_scales(_ptr(scales), _ptr(grad_scales), _ptr(exp_avg), _ptr(exp_avg_sq),
+                                            scales.numel(), int(step), float(lr), float(beta1), float(beta2),
+                                            float(eps), float(weight_decay), _stream(stream)), "sasq_adamw_scales")
 
 
 def sasq_fakequant_per_channel_workspace(T: int, K: int) -> int:

@@ -80,10 +80,52 @@ __global__ void __launch_bounds__(kThreads) quantize_weight_kernel(const float* 
     }
 }
 
+// One AdamW step on the factors (the only trainable parameters, Sec. 4.2 / 5.1), fp32, one thread per factor:
+//   m = b1 m + (1 - b1) g;  v = b2 v + (1 - b2) g^2;  s -= lr * ( (m / c1) / (sqrt(v / c2) + eps) + wd * s )
+// with the bias corrections c1 = 1 - b1^step, c2 = 1 - b2^step computed on the host.
+__global__ void __launch_bounds__(kThreads) adamw_scales_kernel(float* __restrict__ s, const float* __restrict__ g,
+                                                                float* __restrict__ m, float* __restrict__ v, int n,
+                                                                float lr, float b1, float b2, float eps, float wd,
+                                                                float c1, float c2) {
+    const int i = blockIdx.x * kThreads + threadIdx.x;
+    if (i >= n) return;
+    const float gi = g[i];
+    const float mi = __fadd_rn(__fmul_rn(b1, m[i]), __fmul_rn(1.0f - b1, gi));
+    const float vi = __fadd_rn(__fmul_rn(b2, v[i]), __fmul_rn(1.0f - b2, __fmul_rn(gi, gi)));
+    m[i] = mi;
+    v[i] = vi;
+    const float mhat = __fdiv_rn(mi, c1);
+    const float vhat = __fdiv_rn(vi, c2);
+    const float si = s[i];
+    const float upd = __fadd_rn(__fdiv_rn(mhat, __fadd_rn(__fsqrt_rn(vhat), eps)), __fmul_rn(wd, si));
+    s[i] = __fsub_rn(si, __fmul_rn(lr, upd));
+}
+
 }  // namespace
 }  // namespace sasq
 
 extern "C" {
+
+int sasq_adamw_scales(float* scales_dev, const float* grad_scales_dev, float* exp_avg_dev, float* exp_avg_sq_dev,
+                      int n, int step, float lr, float beta1, float beta2, float eps, float weight_decay,
+                      void* stream) {
+    using namespace sasq;
+    if (n < 0 || step < 1) return SASQ_ERR_INVALID_ARG;
+    if (n > 0 && (scales_dev == nullptr || grad_scales_dev == nullptr || exp_avg_dev == nullptr ||
+                  exp_avg_sq_dev == nullptr))
+        return SASQ_ERR_INVALID_ARG;
+    if (!(beta1 >= 0.0f && beta1 < 1.0f) || !(beta2 >= 0.0f && beta2 < 1.0f) || !(eps > 0.0f))
+        return SASQ_ERR_INVALID_ARG;
+    if (n == 0) return SASQ_OK;
+    if (device_sm_count_if_sm100() <= 0) return SASQ_ERR_UNSUPPORTED;
+    double p1 = 1.0, p2 = 1.0;
+    for (int i = 0; i < step; ++i) { p1 *= (double)beta1; p2 *= (double)beta2; }
+    adamw_scales_kernel<<<(n + kThreads - 1) / kThreads, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        scales_dev, grad_scales_dev, exp_avg_dev, exp_avg_sq_dev, n, lr, beta1, beta2, eps, weight_decay,
+        (float)(1.0 - p1), (float)(1.0 - p2));
+    if (cudaGetLastError() != cudaSuccess) return SASQ_ERR_CUDA;
+    return SASQ_OK;
+}
 
 size_t sasq_absmax_scale_workspace(int64_t numel) {
     (void)numel;

@@ -63,7 +63,7 @@ unsigned* next_ticket() {
     return base[dev] + (next.fetch_add(1u, std::memory_order_relaxed) % kTicketSlots);
 }
 
-template <bool BF, bool FWD, bool BWD>
+template <bool BF, bool FWD, bool BWD, int VARIANT = 0>
 cudaError_t launch_stream(const QParams& p, int grid, cudaStream_t st) {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)grid, 1, 1);
@@ -72,14 +72,14 @@ cudaError_t launch_stream(const QParams& p, int grid, cudaStream_t st) {
     cudaLaunchAttribute attr[1] = {pdl_attribute()};
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, fakequant_kernel<BF, FWD, BWD, kThreads, (BWD ? kUnroll : kUnrollFwdOnly), kBlocksPerSM, kLoadHint, kStoreHint>, p);
+    return cudaLaunchKernelEx(&cfg, fakequant_kernel<BF, FWD, BWD, kThreads, (BWD ? kUnroll : kUnrollFwdOnly), kBlocksPerSM, kLoadHint, kStoreHint, VARIANT>, p);
 }
 
-template <bool BF>
+template <bool BF, int VARIANT = 0>
 cudaError_t launch_mode(bool fwd, bool bwd, const QParams& p, int grid, cudaStream_t st) {
-    if (fwd && bwd) return launch_stream<BF, true, true>(p, grid, st);
-    if (fwd) return launch_stream<BF, true, false>(p, grid, st);
-    return launch_stream<BF, false, true>(p, grid, st);
+    if (fwd && bwd) return launch_stream<BF, true, true, VARIANT>(p, grid, st);
+    if (fwd) return launch_stream<BF, true, false, VARIANT>(p, grid, st);
+    return launch_stream<BF, false, true, VARIANT>(p, grid, st);
 }
 
 int grid_for(long long max_numel, int sm_count) {
@@ -91,8 +91,18 @@ int grid_for(long long max_numel, int sm_count) {
     return (int)g;
 }
 
+template <bool BF>
+cudaError_t launch_variant(int variant, bool fwd, bool bwd, const QParams& p, int grid, cudaStream_t st) {
+    if (variant == SASQ_WITHOUT_ROUND) return launch_mode<BF, 1>(fwd, bwd, p, grid, st);
+    if (variant == SASQ_WITHOUT_CLAMP) return launch_mode<BF, 2>(fwd, bwd, p, grid, st);
+    return launch_mode<BF, 0>(fwd, bwd, p, grid, st);
+}
+
 int run_multi(const sasq_qdesc_t* descs, int n_tensors, const float* scales_dev, float* grad_scales_dev,
-              int n_scales, int accumulate, int dt, int bits, void* workspace, size_t ws_bytes, void* stream) {
+              int n_scales, int accumulate, int dt, int bits, void* workspace, size_t ws_bytes, void* stream,
+              int variant = SASQ_FULL_OPERATOR) {
+    if (variant != SASQ_FULL_OPERATOR && variant != SASQ_WITHOUT_ROUND && variant != SASQ_WITHOUT_CLAMP)
+        return SASQ_ERR_INVALID_ARG;
     if (n_tensors < 0 || n_scales <= 0 || (n_tensors > 0 && descs == nullptr)) return SASQ_ERR_INVALID_ARG;
     if (scales_dev == nullptr) return SASQ_ERR_INVALID_ARG;
     if (bits < 2 || bits > 8) return SASQ_ERR_INVALID_ARG;
@@ -155,8 +165,8 @@ int run_multi(const sasq_qdesc_t* descs, int n_tensors, const float* scales_dev,
             p.ticket = next_ticket();
             if (p.ticket == nullptr) return SASQ_ERR_CUDA;
         }
-        cudaError_t e = (dt == SASQ_BF16) ? launch_mode<true>(fwd, bwd, p, grid, st)
-                                          : launch_mode<false>(fwd, bwd, p, grid, st);
+        cudaError_t e = (dt == SASQ_BF16) ? launch_variant<true>(variant, fwd, bwd, p, grid, st)
+                                          : launch_variant<false>(variant, fwd, bwd, p, grid, st);
         if (e != cudaSuccess) return SASQ_ERR_CUDA;
     }
     return SASQ_OK;
@@ -164,7 +174,7 @@ int run_multi(const sasq_qdesc_t* descs, int n_tensors, const float* scales_dev,
 
 int run_single(const void* x, const void* grad_y, void* y, void* grad_x, float* grad_scale_dev, int accumulate,
                int64_t numel, int dt, const float* scale_dev, int bits, void* workspace, size_t ws_bytes,
-               void* stream, bool fwd, bool bwd) {
+               void* stream, bool fwd, bool bwd, int variant = SASQ_FULL_OPERATOR) {
     if (numel < 0) return SASQ_ERR_INVALID_ARG;
     if (scale_dev == nullptr) return SASQ_ERR_INVALID_ARG;
     if (bits < 2 || bits > 8) return SASQ_ERR_INVALID_ARG;
@@ -188,7 +198,7 @@ int run_single(const void* x, const void* grad_y, void* y, void* grad_x, float* 
     d.grad_x = bwd ? grad_x : nullptr;
     d.numel = numel;
     d.scale_index = 0;
-    return run_multi(&d, 1, scale_dev, grad_scale_dev, 1, accumulate, dt, bits, workspace, ws_bytes, stream);
+    return run_multi(&d, 1, scale_dev, grad_scale_dev, 1, accumulate, dt, bits, workspace, ws_bytes, stream, variant);
 }
 
 // ---------------------------------------------------------------------------
@@ -299,6 +309,13 @@ int sasq_fakequant_fwd_bwd(const void* x, const void* grad_y, void* y, void* gra
                            void* workspace, size_t ws_bytes, void* stream) {
     return sasq::run_single(x, grad_y, y, grad_x, grad_scale_dev, accumulate, numel, dt, scale_dev, bits,
                             workspace, ws_bytes, stream, true, true);
+}
+
+int sasq_fakequant_fwd_bwd_ablation(const void* x, const void* grad_y, void* y, void* grad_x, float* grad_scale_dev,
+                                    int accumulate, int64_t numel, int dt, const float* scale_dev, int bits,
+                                    int variant, void* workspace, size_t ws_bytes, void* stream) {
+    return sasq::run_single(x, grad_y, y, grad_x, grad_scale_dev, accumulate, numel, dt, scale_dev, bits, workspace,
+                            ws_bytes, stream, true, true, variant);
 }
 
 int sasq_fakequant_fwd_bwd_multi(const sasq_qdesc_t* descs_host, int n_tensors, const float* scales_dev,

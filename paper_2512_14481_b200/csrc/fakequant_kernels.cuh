@@ -52,23 +52,42 @@ struct Quant2 {
     float p0, p1;    // g * dy/ds
 };
 
-template <bool BF, bool FWD, bool BWD>
+// The operator's two non-linear steps, with the ablations of Table 3: VARIANT 0 = full operator,
+// 1 = "w/o round" (the rounding step is the identity), 2 = "w/o clamp" (the clamp is the identity and always
+// passes the gradient).
+template <int VARIANT>
+__device__ __forceinline__ float step_round(float t) {
+    if constexpr (VARIANT == 1) return t;
+    else return rintf(t);
+}
+template <int VARIANT>
+__device__ __forceinline__ float step_clamp(float r, float qn, float qp) {
+    if constexpr (VARIANT == 2) return r;
+    else return fminf(fmaxf(r, -qn), qp);
+}
+template <int VARIANT>
+__device__ __forceinline__ bool clamp_passes(float c, float r) {
+    if constexpr (VARIANT == 2) return true;
+    else return c == r;                   // false for NaN as well
+}
+
+template <bool BF, bool FWD, bool BWD, int VARIANT>
 __device__ __forceinline__ Quant2 quant_pair(uint32_t xw, uint32_t gw, float s, float inv, float qn, float qp) {
     Quant2 o;
     const float2 xf = widen2<BF>(xw);
     const float t0 = __fmul_rn(xf.x, inv);
     const float t1 = __fmul_rn(xf.y, inv);
-    const float r0 = rintf(t0);
-    const float r1 = rintf(t1);
-    const float c0 = fminf(fmaxf(r0, -qn), qp);
-    const float c1 = fminf(fmaxf(r1, -qn), qp);
+    const float r0 = step_round<VARIANT>(t0);
+    const float r1 = step_round<VARIANT>(t1);
+    const float c0 = step_clamp<VARIANT>(r0, qn, qp);
+    const float c1 = step_clamp<VARIANT>(r1, qn, qp);
     if constexpr (FWD) {
         o.y = narrow2<BF>(__fmul_rn(c0, s), __fmul_rn(c1, s));
     }
     if constexpr (BWD) {
         const float2 gf = widen2<BF>(gw);
-        const bool in0 = (c0 == r0);      // false for NaN as well
-        const bool in1 = (c1 == r1);
+        const bool in0 = clamp_passes<VARIANT>(c0, r0);
+        const bool in1 = clamp_passes<VARIANT>(c1, r1);
         o.dx = (in0 ? (gw & 0x0000FFFFu) : 0u) | (in1 ? (gw & 0xFFFF0000u) : 0u);
         o.p0 = __fmul_rn(gf.x, in0 ? __fsub_rn(r0, t0) : c0);
         o.p1 = __fmul_rn(gf.y, in1 ? __fsub_rn(r1, t1) : c1);
@@ -119,7 +138,7 @@ __device__ __forceinline__ double block_sum_fixed(double v, double* smem /* [THR
     return tot;   // valid in thread 0
 }
 
-template <bool BF, bool FWD, bool BWD, int THREADS, int UNROLL, int MIN_BLOCKS, int LHINT, int SHINT>
+template <bool BF, bool FWD, bool BWD, int THREADS, int UNROLL, int MIN_BLOCKS, int LHINT, int SHINT, int VARIANT = 0>
 __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) fakequant_kernel(const __grid_constant__ QParams p) {
     __shared__ double warp_sums[THREADS / 32];
     pdl_launch_dependents();
@@ -155,7 +174,7 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) fakequant_kernel(const __
                     if constexpr (BWD) { gw[0] = gv[u].x; gw[1] = gv[u].y; gw[2] = gv[u].z; gw[3] = gv[u].w; }
                     Quant2 q[4];
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) q[j] = quant_pair<BF, FWD, BWD>(xw[j], gw[j], s, inv, qn, qp);
+                    for (int j = 0; j < 4; ++j) q[j] = quant_pair<BF, FWD, BWD, VARIANT>(xw[j], gw[j], s, inv, qn, qp);
                     if constexpr (FWD) store16<SHINT>(d.y + v, make_uint4(q[0].y, q[1].y, q[2].y, q[3].y));
                     if constexpr (BWD) {
                         store16<SHINT>(d.dx + v, make_uint4(q[0].dx, q[1].dx, q[2].dx, q[3].dx));
@@ -174,12 +193,12 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) fakequant_kernel(const __
             const uint16_t xh = reinterpret_cast<const uint16_t*>(d.x)[i];
             const float xf = widen1<BF>(xh);
             const float t = __fmul_rn(xf, inv);
-            const float r = rintf(t);
-            const float c = fminf(fmaxf(r, -qn), qp);
+            const float r = step_round<VARIANT>(t);
+            const float c = step_clamp<VARIANT>(r, qn, qp);
             if constexpr (FWD) reinterpret_cast<uint16_t*>(d.y)[i] = narrow1<BF>(__fmul_rn(c, s));
             if constexpr (BWD) {
                 const uint16_t gh = reinterpret_cast<const uint16_t*>(d.g)[i];
-                const bool in = (c == r);
+                const bool in = clamp_passes<VARIANT>(c, r);
                 reinterpret_cast<uint16_t*>(d.dx)[i] = in ? gh : (uint16_t)0;
                 acc += (double)__fmul_rn(widen1<BF>(gh), in ? __fsub_rn(r, t) : c);
             }
