@@ -201,6 +201,21 @@ SASQ_API int sasq_static_w8a8_linear(const void* x, const int8_t* w, const float
                             const void* bias, void* y, int32_t* acc_out, int64_t T, int64_t N, int64_t K,
                             int dt, int bits, void* workspace, size_t ws_bytes, void* stream);
 
+/* Bytes of scratch sasq_dynamic_w8a8_linear needs for this shape. */
+SASQ_API size_t sasq_dynamic_w8a8_linear_workspace(int64_t T, int64_t N, int64_t K);
+
+/* W8A8 linear with DYNAMIC per-token activation factors: the generation phase of the paper's phased quantization
+ * (Sec. 4.4; one token per sequence, so per-token equals per-tensor on that row).  For every row t:
+ *   s_t        = max_k |x[t,k]| / Qp                  (Eq. 1 on the row; an all-zero row takes s_t = 1)
+ *   X_int[t,k] = int8(c(x[t,k])) with s = s_t,   acc[t,n] = sum_k X_int[t,k] * w[n,k]
+ *   y[t,n]     = narrow( fl32(acc) * fl32(s_t * w_scale[n]) (+ bias[n]) )
+ * Arguments as for sasq_static_w8a8_linear, without x_scale_dev.  row_scale_out: [T] fp32 that receives the
+ * factors, or NULL (they are then kept in the workspace).  One extra launch computes the factors and the codes (a
+ * row's factor needs the whole row first). */
+SASQ_API int sasq_dynamic_w8a8_linear(const void* x, const int8_t* w, const float* w_scale, const void* bias, void* y,
+                                      float* row_scale_out, int32_t* acc_out, int64_t T, int64_t N, int64_t K, int dt,
+                                      int bits, void* workspace, size_t ws_bytes, void* stream);
+
 /* How sasq_static_w8a8_linear splits a [T, N] output over `num_pairs` co-operating CTA pairs when T > 128
  * (introspection for tests and tuning; runs on the host, touches no device).  Every 256-row block is cut into the
  * same number of column tiles, widths multiples of 16 that differ by at most 16; the number is chosen so that the

@@ -274,3 +274,25 @@ def adamw_step(s, g, m, v, step: int, lr: float = 2e-4, beta1: float = 0.9, beta
     v_hat = v / (1.0 - beta2 ** step)
     s_new = s - lr * (m_hat / (np.sqrt(v_hat) + eps) + weight_decay * s)
     return s_new, m, v
+
+
+def w8a8_linear_dynamic(x: np.ndarray, tag: int, w_int: np.ndarray, w_scale: np.ndarray, bits: int = 8,
+                        bias: np.ndarray | None = None):
+    """Dynamic per-token W8A8 linear (Sec. 4.4, generation phase): every row is a tensor of its own with the
+    max-based factor of Eq. 1 (an all-zero row takes factor 1), then Eq. 2.  Written as the per-tensor routines
+    applied row by row.  Returns (y bits, acc int32, row factors fp32)."""
+    x = _u16(x)
+    T, K = x.shape
+    N = w_int.shape[0]
+    y = np.zeros((T, N), np.uint16)
+    acc = np.zeros((T, N), np.int32)
+    s_rows = np.zeros(T, np.float32)
+    for t in range(T):
+        row = x[t:t + 1]
+        s = absmax_scale(row, tag, bits)
+        if not s > 0:
+            s = np.float32(1.0)
+        s_rows[t] = s
+        y_t, _, acc_t = w8a8_linear(row, tag, w_int, w_scale, float(s), bits, bias)
+        y[t], acc[t] = y_t[0], acc_t[0]
+    return y, acc, s_rows

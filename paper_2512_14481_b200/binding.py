@@ -21,7 +21,7 @@ __all__ = [
     "sasq_quantize_weight", "linear_launches", "sasq_fakequant_fwd_bwd_static", "sasq_static_w8a8_linear_tiles",
     "sasq_fakequant_per_channel_workspace", "sasq_fakequant_fwd_bwd_per_channel",
     "sasq_fakequant_fwd_bwd_ablation", "sasq_adamw_scales", "SASQ_FULL_OPERATOR", "SASQ_WITHOUT_ROUND",
-    "SASQ_WITHOUT_CLAMP",
+    "SASQ_WITHOUT_CLAMP", "sasq_dynamic_w8a8_linear_workspace", "sasq_dynamic_w8a8_linear",
 ]
 
 SASQ_F16 = 0
@@ -99,6 +99,10 @@ def load_library() -> ctypes.CDLL:
     L.sasq_fakequant_per_channel_workspace.argtypes = [i64, i64]
     L.sasq_fakequant_fwd_bwd_per_channel.restype = i32
     L.sasq_fakequant_fwd_bwd_per_channel.argtypes = [vp, vp, vp, vp, vp, i32, i64, i64, i32, vp, i32, vp, sz, vp]
+    L.sasq_dynamic_w8a8_linear_workspace.restype = sz
+    L.sasq_dynamic_w8a8_linear_workspace.argtypes = [i64, i64, i64]
+    L.sasq_dynamic_w8a8_linear.restype = i32
+    L.sasq_dynamic_w8a8_linear.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, sz, vp]
     L.sasq_static_w8a8_linear_tiles.restype = i32
     L.sasq_static_w8a8_linear_tiles.argtypes = [i64, i64, i32, i32, ctypes.POINTER(ctypes.c_int32), i32]
     L.sasq_device_status.restype = i32
@@ -309,6 +313,36 @@ def sasq_static_w8a8_linear(x, w, w_scale, x_scale, y, bias=None, acc_out=None, 
     _check(load_library().sasq_static_w8a8_linear(_ptr(x), _ptr(w), _ptr(w_scale), _ptr(x_scale), _ptr(bias), _ptr(y),
                                                   _ptr(acc_out), T, N, K, _dt(x), int(bits), _ptr(workspace),
                                                   _nbytes(workspace), _stream(stream)), "sasq_static_w8a8_linear")
+
+
+def sasq_dynamic_w8a8_linear_workspace(T: int, N: int, K: int) -> int:
+    return int(load_library().sasq_dynamic_w8a8_linear_workspace(int(T), int(N), int(K)))
+
+
+def sasq_dynamic_w8a8_linear(x, w, w_scale, y, bias=None, row_scale_out=None, acc_out=None, workspace=None,
+                             bits: int = 8, stream=None) -> None:
+    """Dynamic per-token W8A8 linear: x [T, K], w [N, K] int8, w_scale [N], y [T, N]; row_scale_out [T] fp32 or None."""
+    _dev(x, "x"); _dev(w, "w", torch.int8); _dev(w_scale, "w_scale", torch.float32); _dev(y, "y", x.dtype)
+    for name, t, dtp in (("bias", bias, x.dtype), ("row_scale_out", row_scale_out, torch.float32),
+                         ("acc_out", acc_out, torch.int32)):
+        if t is not None:
+            _dev(t, name, dtp)
+    if workspace is not None:
+        _dev(workspace, "workspace")
+    if x.dim() != 2 or w.dim() != 2 or x.shape[1] != w.shape[1]:
+        raise ValueError("x must be [T, K] and w [N, K]")
+    T, K = x.shape
+    N = w.shape[0]
+    if tuple(y.shape) != (T, N) or w_scale.numel() != N or (bias is not None and bias.numel() != N):
+        raise ValueError("y must be [T, N], w_scale and bias [N]")
+    if row_scale_out is not None and row_scale_out.numel() != T:
+        raise ValueError("row_scale_out must be [T]")
+    if acc_out is not None and tuple(acc_out.shape) != (T, N):
+        raise ValueError("acc_out must be [T, N]")
+    _check(load_library().sasq_dynamic_w8a8_linear(_ptr(x), _ptr(w), _ptr(w_scale), _ptr(bias), _ptr(y),
+                                                   _ptr(row_scale_out), _ptr(acc_out), T, N, K, _dt(x), int(bits),
+                                                   _ptr(workspace), _nbytes(workspace), _stream(stream)),
+           "sasq_dynamic_w8a8_linear")
 
 
 def sasq_static_w8a8_linear_tiles(T: int, N: int, num_pairs: int, pair_id: int):

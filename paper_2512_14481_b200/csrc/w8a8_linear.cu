@@ -55,7 +55,8 @@ constexpr size_t kSmemBytes = 1024 /* alignment slack */ + (size_t)STAGES * STAG
 
 struct LinearParams {
     const float* w_scale;
-    const float* x_scale;
+    const float* x_scale;      // one static factor for the whole tensor, or
+    const float* row_scale;    // [T] one factor per row (dynamic per-token quantization); then x_scale is unused
     const void* bias;
     void* y;
     int32_t* acc_out;
@@ -64,6 +65,12 @@ struct LinearParams {
     int* status;
     long long wait_limit;
 };
+
+// factor of output (t, n): the staged per-channel value already holds s_x * s_w[n] for a static factor; with
+// per-row factors it holds s_w[n] and the row's factor is multiplied in here, fl32(s_row * s_w[n])
+__device__ __forceinline__ float out_scale(bool per_row, float s_row, float staged) {
+    return per_row ? __fmul_rn(s_row, staged) : staged;
+}
 
 // Bounded wait: false (and the abort flag raised) if the phase did not complete in time
 // or another role already gave up.
@@ -209,8 +216,9 @@ w8a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         // ---------------- epilogue (warps 2..5) ----------------
         const int quad = warp & 3;                      // TMEM lane quadrant this warp may read
         const int et = threadIdx.x - 64;                // 0..127
-        const float sx = __ldg(p.x_scale);
-        if (blockIdx.x == 0 && et == 0 && scale_is_bad(sx)) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
+        const bool per_row = p.row_scale != nullptr;
+        const float sx = per_row ? 1.0f : __ldg(p.x_scale);
+        if (!per_row && blockIdx.x == 0 && et == 0 && scale_is_bad(sx)) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
         bool ok = true;
         int it = 0;
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
@@ -235,6 +243,7 @@ w8a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 
             const int row = m_blk * BM + quad * 32 + lane;
             const bool row_ok = row < p.T;
+            const float s_row = (per_row && row_ok) ? __ldg(p.row_scale + row) : 1.0f;
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * BN);
             uint16_t* yrow = reinterpret_cast<uint16_t*>(p.y) + (size_t)row * p.N + n0;
             int32_t* arow = p.acc_out ? p.acc_out + (size_t)row * p.N + n0 : nullptr;
@@ -249,8 +258,10 @@ w8a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         uint32_t o[4];
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
-                            float f0 = __fmul_rn(__int2float_rn((int)v[j + 2 * q]), tail->scale[c + j + 2 * q]);
-                            float f1 = __fmul_rn(__int2float_rn((int)v[j + 2 * q + 1]), tail->scale[c + j + 2 * q + 1]);
+                            float f0 = __fmul_rn(__int2float_rn((int)v[j + 2 * q]),
+                                                 out_scale(per_row, s_row, tail->scale[c + j + 2 * q]));
+                            float f1 = __fmul_rn(__int2float_rn((int)v[j + 2 * q + 1]),
+                                                 out_scale(per_row, s_row, tail->scale[c + j + 2 * q + 1]));
                             if (p.bias != nullptr) {
                                 f0 = __fadd_rn(f0, tail->bias[c + j + 2 * q]);
                                 f1 = __fadd_rn(f1, tail->bias[c + j + 2 * q + 1]);
@@ -680,8 +691,9 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         // ---------------- epilogue (warps 2..5 of both CTAs) ----------------
         const int quad = warp & 3;
         const int et = threadIdx.x - 64;
-        const float sx = __ldg(p.x_scale);
-        if (blockIdx.x == 0 && et == 0 && scale_is_bad(sx)) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
+        const bool per_row = p.row_scale != nullptr;
+        const float sx = per_row ? 1.0f : __ldg(p.x_scale);
+        if (!per_row && blockIdx.x == 0 && et == 0 && scale_is_bad(sx)) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
         const bool has_bias = p.bias != nullptr;
         bool ok = true;
         int it = 0;
@@ -712,6 +724,7 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             const int row0 = m_blk * PBM + (int)rank * 128 + quad * 32;
             const int row = row0 + lane;
             const bool row_ok = row < p.T;
+            const float s_row = (per_row && row_ok) ? __ldg(p.row_scale + row) : 1.0f;
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * 256);
             int32_t* arow = p.acc_out ? p.acc_out + (size_t)row * p.N + n0 : nullptr;
             uint8_t* my_stage = out_stage + (size_t)quad * 2 * P_OUT_BUF_BYTES;
@@ -733,8 +746,9 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                         uint32_t o[4];
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
-                            float f0 = __fmul_rn(__int2float_rn((int)v[j + 2 * q]), sc[j + 2 * q]);
-                            float f1 = __fmul_rn(__int2float_rn((int)v[j + 2 * q + 1]), sc[j + 2 * q + 1]);
+                            float f0 = __fmul_rn(__int2float_rn((int)v[j + 2 * q]), out_scale(per_row, s_row, sc[j + 2 * q]));
+                            float f1 = __fmul_rn(__int2float_rn((int)v[j + 2 * q + 1]),
+                                                 out_scale(per_row, s_row, sc[j + 2 * q + 1]));
                             if (has_bias) {
                                 f0 = __fadd_rn(f0, bi[j + 2 * q]);
                                 f1 = __fadd_rn(f1, bi[j + 2 * q + 1]);
@@ -774,8 +788,9 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                     uint32_t o[4];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
-                        float f0 = __fmul_rn(__int2float_rn((int)v[j + 2 * q]), sc[j + 2 * q]);
-                        float f1 = __fmul_rn(__int2float_rn((int)v[j + 2 * q + 1]), sc[j + 2 * q + 1]);
+                        float f0 = __fmul_rn(__int2float_rn((int)v[j + 2 * q]), out_scale(per_row, s_row, sc[j + 2 * q]));
+                        float f1 = __fmul_rn(__int2float_rn((int)v[j + 2 * q + 1]),
+                                                 out_scale(per_row, s_row, sc[j + 2 * q + 1]));
                         if (has_bias) {
                             f0 = __fadd_rn(f0, bi[j + 2 * q]);
                             f1 = __fadd_rn(f1, bi[j + 2 * q + 1]);
@@ -935,7 +950,8 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
     const uint32_t tmem_base = tail->tmem_base;
     pdl_wait();                         // set-up done; from here on global memory of earlier kernels is used
 
-    const unsigned items_total = (unsigned)(((long long)p.T * p.K) >> 4);      // 16 elements each
+    // 16-element items the in-kernel quantizer has to publish (none if the activations came quantized)
+    const unsigned items_total = dp.x != nullptr ? (unsigned)(((long long)p.T * p.K) >> 4) : 0u;
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
@@ -950,7 +966,7 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
                 ptx::mbar_arrive_expect_tx(&tail->full[i], (uint32_t)stage_bytes);
                 ptx::tma_load_2d(ring + (size_t)i * stage_bytes, &tmap_w, &tail->full[i], (kb_begin + i) * BK, n0);
             }
-            {
+            if (items_total != 0) {
                 const long long t0 = clock64();
                 int polls = 0;
                 for (;;) {
@@ -1018,9 +1034,10 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
     } else {
         // ---------------- activation quantizer, then epilogue (warps 2..5) ----------------
         const int et = threadIdx.x - 64;                       // 0..127
-        const float sx = __ldg(p.x_scale);
-        if (blockIdx.x == 0 && et == 0 && scale_is_bad(sx)) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
-        {
+        const bool per_row = p.row_scale != nullptr;
+        const float sx = per_row ? 1.0f : __ldg(p.x_scale);
+        if (!per_row && blockIdx.x == 0 && et == 0 && scale_is_bad(sx)) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
+        if (dp.x != nullptr) {
             const float inv = __fdiv_rn(1.0f, sx);
             const uint4* src = reinterpret_cast<const uint4*>(dp.x);
             uint4* dst = reinterpret_cast<uint4*>(dp.a_int8);
@@ -1080,7 +1097,8 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
         const int rows = 128 / dp.split;
         const int pstride = dp.tp + 4;
         const bool has_bias = p.bias != nullptr;
-        const float sx = __ldg(p.x_scale);
+        const bool per_row = p.row_scale != nullptr;
+        const float sx = per_row ? 1.0f : __ldg(p.x_scale);
         const int items = rows * (dp.tp >> 2);
         for (int it = et; it < items; it += 128) {
             const int n_local = rank * rows + (it % rows);
@@ -1096,13 +1114,15 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
                 acc[0] += v0; acc[1] += v1; acc[2] += v2; acc[3] += v3;
             }
             if (n < p.N) {
-                const float sc = __fmul_rn(sx, __ldg(p.w_scale + n));
+                const float ws = __ldg(p.w_scale + n);
+                const float sc = __fmul_rn(sx, ws);
                 const float bv = has_bias ? widen1<BF>(__ldg(reinterpret_cast<const uint16_t*>(p.bias) + n)) : 0.0f;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const int t = t0 + j;
                     if (t < p.T) {
-                        float f = __fmul_rn(__int2float_rn(acc[j]), sc);
+                        const float sct = per_row ? __fmul_rn(__ldg(p.row_scale + t), ws) : sc;
+                        float f = __fmul_rn(__int2float_rn(acc[j]), sct);
                         if (has_bias) f = __fadd_rn(f, bv);
                         reinterpret_cast<uint16_t*>(p.y)[(size_t)t * p.N + n] = narrow1<BF>(f);
                         if (p.acc_out != nullptr) p.acc_out[(size_t)t * p.N + n] = acc[j];
@@ -1122,7 +1142,7 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
         ptx::tmem_dealloc(tmem_base, dp.tmem_cols);
     }
     // the CTA that finishes last leaves the counters at zero for the next launch that draws them
-    if (threadIdx.x == 0) {
+    if (dp.x != nullptr && threadIdx.x == 0) {
         if (atomicAdd(dp.done, 1u) == gridDim.x - 1) {
             *dp.ready = 0u;
             *dp.done = 0u;
@@ -1140,6 +1160,48 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const uint4* __restri
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += stride)
         out[i] = quantize8<BF, false>(x[i], inv, qn, qp);
+}
+
+// Dynamic per-token quantization (Sec. 4.4, generation phase): one block per row of x.  The row's factor is its
+// own max-based one, s_t = max_k |x[t,k]| / Qp (Eq. 1; an all-zero row takes s_t = 1), then the row is quantized with
+// it exactly like the static path: code = clamp(rint(x * fl32(1 / s_t))).  The row is read twice; the second read
+// comes from L2.
+template <bool BF>
+__global__ void __launch_bounds__(256) quantize_rows_dynamic_kernel(const uint4* __restrict__ x, uint2* __restrict__ out,
+                                                                    float* __restrict__ row_scale, int K, float qn,
+                                                                    float qp) {
+    __shared__ float warp_max[8];
+    __shared__ float s_inv;
+    pdl_launch_dependents();
+    pdl_wait();
+    const int vec = K >> 3;
+    const uint4* row = x + (size_t)blockIdx.x * vec;
+    float m = 0.0f;
+    for (int i = threadIdx.x; i < vec; i += 256) {
+        const uint4 v = row[i];
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const float2 f = widen2<BF>(w[q]);
+            m = fmaxf(m, fmaxf(fabsf(f.x), fabsf(f.y)));
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, off));
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float mm = 0.0f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) mm = fmaxf(mm, warp_max[w]);
+        const float sc = mm > 0.0f ? __fdiv_rn(mm, qp) : 1.0f;
+        row_scale[blockIdx.x] = sc;
+        s_inv = __fdiv_rn(1.0f, sc);
+    }
+    __syncthreads();
+    const float inv = s_inv;
+    uint2* orow = out + (size_t)blockIdx.x * vec;
+    for (int i = threadIdx.x; i < vec; i += 256) orow[i] = quantize8<BF, false>(row[i], inv, qn, qp);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -1396,22 +1458,30 @@ size_t sasq_static_w8a8_linear_workspace(int64_t T, int64_t N, int64_t K) {
     return (size_t)(((T * K + 15) / 16) * 16 + 256);
 }
 
-int sasq_static_w8a8_linear(const void* x, const int8_t* w, const float* w_scale, const float* x_scale_dev,
-                            const void* bias, void* y, int32_t* acc_out, int64_t T, int64_t N, int64_t K, int dt,
-                            int bits, void* workspace, size_t ws_bytes, void* stream) {
-    using namespace sasq;
+}  // extern "C"
+
+namespace sasq {
+namespace {
+
+// dynamic == false: static factor x_scale_dev (the hot path).  dynamic == true: every row gets its own max-based
+// factor, written to row_scale_out (or to the workspace when that is NULL) by a launch that also quantizes the rows.
+int linear_impl(const void* x, const int8_t* w, const float* w_scale, const float* x_scale_dev, bool dynamic,
+                float* row_scale_out, const void* bias, void* y, int32_t* acc_out, int64_t T, int64_t N, int64_t K,
+                int dt, int bits, void* workspace, size_t ws_bytes, void* stream) {
     if (T < 0 || N <= 0 || K <= 0) return SASQ_ERR_INVALID_ARG;
     if (dt != SASQ_F16 && dt != SASQ_BF16) return SASQ_ERR_INVALID_ARG;
     if (bits < 2 || bits > 8) return SASQ_ERR_INVALID_ARG;
-    if (w == nullptr || w_scale == nullptr || x_scale_dev == nullptr) return SASQ_ERR_INVALID_ARG;
+    if (w == nullptr || w_scale == nullptr || (!dynamic && x_scale_dev == nullptr)) return SASQ_ERR_INVALID_ARG;
     if (T > 0 && (x == nullptr || y == nullptr)) return SASQ_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(row_scale_out) & 3u) return SASQ_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(acc_out) ||
         (reinterpret_cast<uintptr_t>(w_scale) & 3u) || (reinterpret_cast<uintptr_t>(bias) & 1u))
         return SASQ_ERR_INVALID_ARG;
     if (K % 16 != 0 || N % 8 != 0 || K > 131072 || T > (1 << 24) || N > (1 << 24)) return SASQ_ERR_UNSUPPORTED;
     if (T == 0) return SASQ_OK;
-    if (workspace == nullptr || !aligned16(workspace) || ws_bytes < sasq_static_w8a8_linear_workspace(T, N, K))
-        return SASQ_ERR_WORKSPACE;
+    const size_t ws_need = dynamic ? sasq_dynamic_w8a8_linear_workspace(T, N, K)
+                                   : sasq_static_w8a8_linear_workspace(T, N, K);
+    if (workspace == nullptr || !aligned16(workspace) || ws_bytes < ws_need) return SASQ_ERR_WORKSPACE;
     const int sm_count = device_sm_count_if_sm100();
     if (sm_count <= 0) return SASQ_ERR_UNSUPPORTED;
     int* status = status_word_ptr();
@@ -1427,8 +1497,32 @@ int sasq_static_w8a8_linear(const void* x, const int8_t* w, const float* w_scale
     const int n_tiles128 = (int)((N + 127) / 128);
     const int split = (T <= BM && n_tiles128 <= sm_count)
                           ? decode_split(dt == SASQ_BF16, n_tiles128, k_blocks, sm_count, kDecodeSmem) : 0;
-    const bool in_kernel_quantizer = split > 0 || (T > BM && (T + PBM - 1) / PBM <= kMaxRowBlocks);
-    if (!in_kernel_quantizer) {
+    const bool in_kernel_quantizer = !dynamic && (split > 0 || (T > BM && (T + PBM - 1) / PBM <= kMaxRowBlocks));
+    const float* row_scale = nullptr;
+    if (dynamic) {
+        // per-token factors and codes by a launch of their own (the factor of a row needs the whole row first)
+        float* rs = row_scale_out;
+        if (rs == nullptr) {
+            const uintptr_t after = reinterpret_cast<uintptr_t>(a_int8) + (uintptr_t)((T * K + 255) / 256 * 256);
+            rs = reinterpret_cast<float*>(after);
+        }
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((unsigned)T, 1, 1);
+        cfg.blockDim = dim3(256, 1, 1);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1] = {pdl_attribute()};
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaError_t qe;
+        if (dt == SASQ_BF16)
+            qe = cudaLaunchKernelEx(&cfg, quantize_rows_dynamic_kernel<true>, static_cast<const uint4*>(x),
+                                    reinterpret_cast<uint2*>(a_int8), rs, (int)K, qn, qp);
+        else
+            qe = cudaLaunchKernelEx(&cfg, quantize_rows_dynamic_kernel<false>, static_cast<const uint4*>(x),
+                                    reinterpret_cast<uint2*>(a_int8), rs, (int)K, qn, qp);
+        if (qe != cudaSuccess) return SASQ_ERR_CUDA;
+        row_scale = rs;
+    } else if (!in_kernel_quantizer) {
         const long long n8 = (T * K) / 8;     // K % 16 == 0
         long long blocks = (n8 + 255) / 256;
         if (blocks > (long long)sm_count * 8) blocks = (long long)sm_count * 8;
@@ -1447,6 +1541,7 @@ int sasq_static_w8a8_linear(const void* x, const int8_t* w, const float* w_scale
     LinearParams p{};
     p.w_scale = w_scale;
     p.x_scale = x_scale_dev;
+    p.row_scale = row_scale;
     p.bias = bias;
     p.y = y;
     p.acc_out = acc_out;
@@ -1469,11 +1564,13 @@ int sasq_static_w8a8_linear(const void* x, const int8_t* w, const float* w_scale
         dp.n_tiles = n_tiles128;
         dp.tmem_cols = 32;
         while ((int)dp.tmem_cols < dp.tp) dp.tmem_cols <<= 1;
-        dp.x = static_cast<const uint16_t*>(x);
         dp.a_int8 = a_int8;
         dp.qn = qn;
         dp.qp = qp;
-        if (!next_ready_slot(&dp.ready, &dp.done)) return SASQ_ERR_CUDA;
+        if (in_kernel_quantizer) {
+            dp.x = static_cast<const uint16_t*>(x);
+            if (!next_ready_slot(&dp.ready, &dp.done)) return SASQ_ERR_CUDA;
+        }
         if (!make_tmap(&tmap_w, w, N, K, 128) || !make_tmap(&tmap_a, a_int8, T, K, dp.tp)) return SASQ_ERR_CUDA;
         cudaLaunchConfig_t cfg{};
         cfg.gridDim = dim3((unsigned)(n_tiles128 * split), 1, 1);
@@ -1540,6 +1637,31 @@ int sasq_static_w8a8_linear(const void* x, const int8_t* w, const float* w_scale
     }
     if (cudaGetLastError() != cudaSuccess) return SASQ_ERR_CUDA;
     return SASQ_OK;
+}
+
+}  // namespace
+}  // namespace sasq
+
+extern "C" {
+
+int sasq_static_w8a8_linear(const void* x, const int8_t* w, const float* w_scale, const float* x_scale_dev,
+                            const void* bias, void* y, int32_t* acc_out, int64_t T, int64_t N, int64_t K, int dt,
+                            int bits, void* workspace, size_t ws_bytes, void* stream) {
+    return sasq::linear_impl(x, w, w_scale, x_scale_dev, false, nullptr, bias, y, acc_out, T, N, K, dt, bits,
+                             workspace, ws_bytes, stream);
+}
+
+size_t sasq_dynamic_w8a8_linear_workspace(int64_t T, int64_t N, int64_t K) {
+    if (T <= 0 || K <= 0) return 0;
+    // int8 codes, then one fp32 factor per row
+    return sasq_static_w8a8_linear_workspace(T, N, K) + 256 + (size_t)T * sizeof(float) + 256;
+}
+
+int sasq_dynamic_w8a8_linear(const void* x, const int8_t* w, const float* w_scale, const void* bias, void* y,
+                             float* row_scale_out, int32_t* acc_out, int64_t T, int64_t N, int64_t K, int dt, int bits,
+                             void* workspace, size_t ws_bytes, void* stream) {
+    return sasq::linear_impl(x, w, w_scale, nullptr, true, row_scale_out, bias, y, acc_out, T, N, K, dt, bits,
+                             workspace, ws_bytes, stream);
 }
 
 }  // extern "C"

@@ -178,3 +178,29 @@ def test_grouped_form_reduces_to_eq2_and_matches_float64_eq3(tag):
         codes = oracle.quantize_act(np.ascontiguousarray(x[:, sl]), tag, float(sg[gi]))
         ref += float(sg[gi]) * (codes.astype(np.int64) @ w_int[:, sl].astype(np.int64).T) * ws[None, :].astype(np.float64)
     assert np.all(np.abs(y32 - ref) <= 1e-5 * np.abs(ref).max())
+
+
+def test_dynamic_per_token_linear_against_numpy_on_small_inputs():
+    """Sec. 4.4 generation phase: every row has its own max-based factor.  Checked against the definition typed in
+    numpy float32 / int64 (power-of-two-free data, so rounding decisions are generic), plus the all-zero row."""
+    rng = np.random.default_rng(11)
+    T, K, N = 5, 48, 24
+    x = (rng.normal(0, 2, (T, K))).astype(np.float32)
+    x[3] = 0.0
+    xb = oracle.bits_of(torch.from_numpy(x).to(torch.bfloat16))[0]
+    xw = oracle.widen(xb, oracle.BF16)                      # the bf16 values as float32
+    w_int = rng.integers(-127, 128, (N, K)).astype(np.int8)
+    w_scale = rng.uniform(1e-3, 2e-3, N).astype(np.float32)
+    y, acc, s = oracle.w8a8_linear_dynamic(xb, oracle.BF16, w_int, w_scale)
+    for t in range(T):
+        amax = np.abs(xw[t]).max()
+        st = np.float32(amax) / np.float32(127) if amax > 0 else np.float32(1)
+        assert s[t] == st
+        inv = np.float32(1) / st
+        codes = np.clip(np.rint((xw[t] * inv).astype(np.float32)), -128, 127).astype(np.int64)
+        a = codes @ w_int.astype(np.int64).T
+        assert np.array_equal(acc[t], a)
+        y32 = a.astype(np.float32) * (st * w_scale).astype(np.float32)
+        assert np.array_equal(y[t], oracle.narrow(y32.astype(np.float32), oracle.BF16))
+    assert not acc[3].any() and np.abs(np.clip(acc, None, None)).max() > 0
+    assert np.abs(oracle.quantize_act(xb[0:1], oracle.BF16, float(s[0]), 8)).max() == 127     # the row maximum maps to Qp
