@@ -1,0 +1,52 @@
+"""Host logic of the CTA-pair GEMM's work split (runs without a GPU): whatever T, N and the number of resident pairs,
+the tiles of all pairs cover every 256-row block x 16-column unit exactly once, widths are multiples of 16 within
+[16, 256] that differ by at most 16, and no pair gets more than one tile above the average."""
+import itertools
+
+import pytest
+
+import paper_2512_14481_b200 as P
+
+
+def all_tiles(T, N, pairs):
+    return [P.sasq_static_w8a8_linear_tiles(T, N, pairs, p) for p in range(pairs)]
+
+
+@pytest.mark.parametrize("T,N", [(129, 8), (256, 4096), (257, 1024), (300, 776), (2048, 4096), (2048, 11008),
+                                 (4096, 5120), (4096, 13824), (8192, 4096), (8192, 11008), (16384, 4096),
+                                 (1000, 264), (513, 24)])
+@pytest.mark.parametrize("pairs", [74, 66, 1, 7])
+def test_tiles_cover_the_output_exactly_once(T, N, pairs):
+    per_pair = all_tiles(T, N, pairs)
+    row_blocks, units = (T + 255) // 256, (N + 15) // 16
+    seen = set()
+    widths = set()
+    for tiles in per_pair:
+        for row0, col0, width in tiles:
+            assert row0 % 256 == 0 and col0 % 16 == 0 and width % 16 == 0 and 16 <= width <= 256
+            widths.add(width)
+            for u in range(col0 // 16, (col0 + width) // 16):
+                key = (row0 // 256, u)
+                assert key not in seen
+                seen.add(key)
+    assert len(seen) == row_blocks * units
+    assert max(widths) - min(widths) <= 16
+    counts = [len(t) for t in per_pair]
+    assert max(counts) - min(counts) <= 1
+
+
+def test_llama_shapes_fill_the_waves():
+    # columns a pair has to compute vs the ideal share: within 9 % for the benchmark's shapes on 74 pairs (2048 x 4096
+    # has 8 row blocks x 18 tiles = 144 tiles for 148 slots, two tiles of up to 240 columns per pair)
+    for T, N in [(2048, 4096), (2048, 11008), (8192, 4096), (8192, 11008)]:
+        per_pair = all_tiles(T, N, 74)
+        most = max(sum(w for _, _, w in tiles) for tiles in per_pair)
+        ideal = ((T + 255) // 256) * N / 74
+        assert most <= 1.09 * ideal, (T, N, most, ideal)
+
+
+def test_invalid_arguments():
+    lib = P.load_library()
+    assert lib.sasq_static_w8a8_linear_tiles(0, 8, 4, 0, None, 0) == -1
+    assert lib.sasq_static_w8a8_linear_tiles(256, 8, 4, 4, None, 0) == -1
+    assert lib.sasq_static_w8a8_linear_tiles(256, 8, 0, 0, None, 0) == -1
