@@ -851,9 +851,9 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
 // operands are swapped: 128 rows of W are the M side of the MMA (every instruction consumes 4 KB of weights), the
 // T activation rows, padded to a multiple of 16, are the N side, and the accumulator tile in TMEM is
 // [128 output channels x T tokens].  To occupy the whole chip a cluster of S CTAs shares one 128-channel tile and
-// splits K; each CTA parks its partial accumulators in its own shared memory, and after a cluster barrier CTA r
-// adds the S partials of its 128 / S channels through distributed shared memory (int32: exact in any order),
-// dequantises and stores them.
+// splits K; each CTA sends its partial accumulators through distributed shared memory to the CTA that owns the
+// channels (CTA r owns 128 / S of them), and after one cluster barrier every CTA adds the S partials of its channels
+// (int32: exact in any order), dequantises and stores them.
 //   warp 0      TMA producer: W tile (128 x 128 B) + int8 activation tile (TP x 128 B) per stage
 //   warp 1      MMA issuer
 //   warps 2..5  first the activation quantizer (Eq. 1 with the fixed factor, all CTAs share the T x K elements and
@@ -881,6 +881,8 @@ struct DecodeParams {
     int split;           // CTAs per cluster = K slices
     int n_tiles;         // 128-channel tiles
     uint32_t tmem_cols;  // power of two >= max(32, tp)
+    int slots_offset;    // byte offset of the reduction slots in the CTA's shared memory: behind the stages, never
+                         // under them, because peers write there while this CTA may still be in its mainloop
     const uint16_t* x;
     uint8_t* a_int8;
     unsigned* ready;     // [1] 16-element items quantized and visible; zero at launch
@@ -1056,17 +1058,23 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
             if (lane == 0 && mine != 0) atomicAdd(dp.ready, mine);
         }
 
-        // epilogue part 1: this CTA's partial accumulators, TMEM -> own shared memory (over the drained ring),
-        // rows = channels, tp + 4 words apart: 128-bit accesses stay aligned and eight consecutive rows cover
-        // all banks, so neither these stores nor the reads below conflict
+        // epilogue part 1: this CTA's partial accumulators go from TMEM straight into the shared memory of the CTA
+        // that will reduce them (remote stores through distributed shared memory, into slots behind the pipeline stages).  CTA r
+        // owns channels [r * 128 / S, (r + 1) * 128 / S) of the tile and holds one slot per K slice:
+        // [S slots][128 / S channels][tp + 4 words]; rows tp + 4 words apart keep 128-bit accesses aligned and
+        // let eight consecutive rows cover all banks.
         const int quad = warp & 3;                              // TMEM lane quadrant of this warp
         const int pstride = dp.tp + 4;
-        int32_t* part = reinterpret_cast<int32_t*>(ring);
+        const int rows = 128 / dp.split;
         bool ok = wait_bounded_d(&tail->acc_full, 0u, tail, p);
         ok = epilogue_all_ok(ok);
         if (ok) {
             ptx::tc_fence_after_sync();
-            uint4* prow = reinterpret_cast<uint4*>(part + (size_t)(quad * 32 + lane) * pstride);
+            const int n_local = quad * 32 + lane;
+            const int owner = n_local / rows;
+            const uint32_t local = ptx::smem_u32(ring) + (uint32_t)dp.slots_offset +
+                                   (uint32_t)((rank * rows + (n_local - owner * rows)) * pstride) * 4u;
+            const uint32_t dst = ptx::mapa_u32(local, (uint32_t)owner);
             if (kb_end > kb_begin) {
                 const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
                 for (int c = 0; c < dp.tp; c += 16) {
@@ -1075,24 +1083,29 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
                     ptx::tmem_ld_wait();
 #pragma unroll
                     for (int j = 0; j < 4; ++j)
-                        prow[(c >> 2) + j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                        asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (uint32_t)(c + 4 * j) * 4u),
+                                     "r"(v[4 * j]), "r"(v[4 * j + 1]), "r"(v[4 * j + 2]), "r"(v[4 * j + 3]) : "memory");
                 }
             } else {
-                for (int c = 0; c < dp.tp; c += 4) prow[c >> 2] = make_uint4(0u, 0u, 0u, 0u);
+                for (int c = 0; c < dp.tp; c += 4)
+                    asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(dst + (uint32_t)c * 4u), "r"(0u)
+                                 : "memory");
             }
         }
         ptx::tc_fence_before_sync();
     }
 
-    // every CTA's partials are in place (or the launch has been abandoned: a role gave up after a bounded wait and
-    // the status word says so; the sums below are then garbage but every access stays in bounds)
+    // every CTA's partials are in their owner's shared memory after this barrier (or the launch has been abandoned:
+    // a role gave up after a bounded wait and the status word says so; the sums below are then garbage but every
+    // access stays in bounds).  Nobody touches another CTA's shared memory afterwards, so the CTAs may finish
+    // independently.
     __syncthreads();
     ptx::cluster_sync_all();
 
     if (warp >= 2) {
-        // epilogue part 2: CTA r reduces channels [r * 128 / S, (r + 1) * 128 / S) of the tile over the S partials.
-        // One work item = one channel x four consecutive tokens (one 128-bit read per partial); consecutive
-        // threads take consecutive channels so that the 16-bit stores of one token coalesce.
+        // epilogue part 2: add the S slots of this CTA's channels, dequantise, store.  One work item = one channel
+        // x four consecutive tokens (one 128-bit read per slot); consecutive threads take consecutive channels so
+        // that the 16-bit stores of one token coalesce.
         const int et = threadIdx.x - 64;
         const int rows = 128 / dp.split;
         const int pstride = dp.tp + 4;
@@ -1100,18 +1113,15 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
         const bool per_row = p.row_scale != nullptr;
         const float sx = per_row ? 1.0f : __ldg(p.x_scale);
         const int items = rows * (dp.tp >> 2);
+        const int32_t* slots = reinterpret_cast<const int32_t*>(ring + dp.slots_offset);
         for (int it = et; it < items; it += 128) {
-            const int n_local = rank * rows + (it % rows);
+            const int r_local = it % rows;
             const int t0 = (it / rows) << 2;
-            const int n = n0 + n_local;
-            const uint32_t my = ptx::smem_u32(ring) + (uint32_t)(n_local * pstride + t0) * 4u;
+            const int n = n0 + rank * rows + r_local;
             int32_t acc[4] = {0, 0, 0, 0};
             for (int r = 0; r < dp.split; ++r) {
-                int32_t v0, v1, v2, v3;
-                const uint32_t addr = ptx::mapa_u32(my, (uint32_t)r);
-                asm volatile("ld.shared::cluster.v4.s32 {%0, %1, %2, %3}, [%4];"
-                             : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3) : "r"(addr) : "memory");
-                acc[0] += v0; acc[1] += v1; acc[2] += v2; acc[3] += v3;
+                const int4 v = *reinterpret_cast<const int4*>(slots + (size_t)(r * rows + r_local) * pstride + t0);
+                acc[0] += v.x; acc[1] += v.y; acc[2] += v.z; acc[3] += v.w;
             }
             if (n < p.N) {
                 const float ws = __ldg(p.w_scale + n);
@@ -1133,10 +1143,8 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
     }
 
     // ---------------- teardown ----------------
-    // no CTA may leave while a peer can still read its partials
     ptx::tc_fence_before_sync();
     __syncthreads();
-    ptx::cluster_sync_all();
     if (warp == 1) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, dp.tmem_cols);
@@ -1559,7 +1567,10 @@ int linear_impl(const void* x, const int8_t* w, const float* w_scale, const floa
         dp.lp = p;
         dp.tp = (int)((T + 15) / 16) * 16;
         const int stage_bytes = D_W_BYTES + dp.tp * BK;
-        dp.stages = D_RING_BYTES / stage_bytes < D_MAX_STAGES ? D_RING_BYTES / stage_bytes : D_MAX_STAGES;
+        const int slot_bytes = (128 * (dp.tp + 4) * 4 + 1023) & ~1023;          // S x (128 / S) rows of tp + 4 words
+        const int ring_bytes = D_RING_BYTES - slot_bytes;
+        dp.slots_offset = ring_bytes;
+        dp.stages = ring_bytes / stage_bytes < D_MAX_STAGES ? ring_bytes / stage_bytes : D_MAX_STAGES;
         dp.split = split;
         dp.n_tiles = n_tiles128;
         dp.tmem_cols = 32;
