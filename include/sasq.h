@@ -255,6 +255,13 @@ SASQ_API int sasq_adamw_scales(float* scales_dev, const float* grad_scales_dev, 
                                float* exp_avg_sq_dev, int n, int step, float lr, float beta1, float beta2, float eps,
                                float weight_decay, void* stream);
 
+/* Test hook.  Every wait inside the GEMM kernels (on an mbarrier, on the activation quantizer's counters) gives up
+ * after this many SM clock cycles, raises SASQ_ERR_TIMEOUT in the status word and lets the kernel finish in an
+ * orderly way (outputs are then unspecified).  The default is 2^31 cycles, about a second; a negative value restores
+ * it.  Returns the previous limit.  Applies to launches made afterwards.  sasq_device_status clears the library's
+ * internal counters when it reports a timeout, so the next call starts clean. */
+SASQ_API long long sasq_debug_set_wait_limit(long long cycles);
+
 /* Synchronises `stream`, returns the sticky device status word of the current
  * device (SASQ_OK, SASQ_ERR_BAD_SCALE or SASQ_ERR_TIMEOUT) and clears it. */
 SASQ_API int sasq_device_status(void* stream);

@@ -21,7 +21,7 @@ __all__ = [
     "sasq_quantize_weight", "linear_launches", "sasq_fakequant_fwd_bwd_static", "sasq_static_w8a8_linear_tiles",
     "sasq_fakequant_per_channel_workspace", "sasq_fakequant_fwd_bwd_per_channel",
     "sasq_fakequant_fwd_bwd_ablation", "sasq_adamw_scales", "SASQ_FULL_OPERATOR", "SASQ_WITHOUT_ROUND",
-    "SASQ_WITHOUT_CLAMP", "sasq_dynamic_w8a8_linear_workspace", "sasq_dynamic_w8a8_linear",
+    "SASQ_WITHOUT_CLAMP", "sasq_dynamic_w8a8_linear_workspace", "sasq_dynamic_w8a8_linear", "sasq_debug_set_wait_limit",
 ]
 
 SASQ_F16 = 0
@@ -103,6 +103,8 @@ def load_library() -> ctypes.CDLL:
     L.sasq_dynamic_w8a8_linear_workspace.argtypes = [i64, i64, i64]
     L.sasq_dynamic_w8a8_linear.restype = i32
     L.sasq_dynamic_w8a8_linear.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, sz, vp]
+    L.sasq_debug_set_wait_limit.restype = ctypes.c_longlong
+    L.sasq_debug_set_wait_limit.argtypes = [ctypes.c_longlong]
     L.sasq_static_w8a8_linear_tiles.restype = i32
     L.sasq_static_w8a8_linear_tiles.argtypes = [i64, i64, i32, i32, ctypes.POINTER(ctypes.c_int32), i32]
     L.sasq_device_status.restype = i32
@@ -354,6 +356,11 @@ def sasq_static_w8a8_linear_tiles(T: int, N: int, num_pairs: int, pair_id: int):
     buf = (ctypes.c_int32 * (3 * max(n, 1)))()
     L.sasq_static_w8a8_linear_tiles(int(T), int(N), int(num_pairs), int(pair_id), buf, n)
     return [(buf[3 * i], buf[3 * i + 1], buf[3 * i + 2]) for i in range(n)]
+
+
+def sasq_debug_set_wait_limit(cycles: int) -> int:
+    """Test hook: clock cycles after which a wait inside the GEMM kernels gives up (negative restores the default)."""
+    return int(load_library().sasq_debug_set_wait_limit(int(cycles)))
 
 
 def sasq_device_status(stream=None) -> int:

@@ -21,7 +21,13 @@
 namespace sasq {
 
 SASQ_DEFINE_STATUS_WORD(g_linear_status)
-int linear_status_read_and_clear(cudaStream_t st) { return g_linear_status_read_and_clear(st); }
+void linear_reset_counters(cudaStream_t st);
+int linear_status_read_and_clear(cudaStream_t st) {
+    const int status = g_linear_status_read_and_clear(st);
+    // a launch that gave up after a bounded wait may have left its readiness counters half counted: start clean
+    if (status == SASQ_ERR_TIMEOUT) linear_reset_counters(st);
+    return status;
+}
 
 namespace {
 
@@ -39,6 +45,7 @@ constexpr int NUM_THREADS = 192;
 constexpr int EPI_THREADS = 128;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr long long kWaitLimit = 1LL << 31;   // clock cycles a single wait may take (about a second)
+std::atomic<long long> g_wait_limit{kWaitLimit};   // what launches use; tests shorten it to see the give-up path
 
 struct SharedTail {
     uint64_t full[STAGES];
@@ -79,7 +86,7 @@ __device__ __forceinline__ bool wait_bounded(uint64_t* bar, uint32_t parity, Sha
     const long long t0 = clock64();
     int polls = 0;
     while (!ptx::mbar_try_wait(bar, parity)) {
-        if ((++polls & 63) == 0) {
+        if (p.wait_limit <= 0 || (++polls & 63) == 0) {      // a zero limit gives up at the first unsuccessful poll
             if (tail->abort_flag) return false;
             if (clock64() - t0 > p.wait_limit) {
                 tail->abort_flag = 1;
@@ -471,7 +478,7 @@ __device__ __forceinline__ bool wait_rows_ready(const unsigned* counter, unsigne
         unsigned v;
         asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
         if (v >= need) return true;
-        if ((++polls & 15) == 0) {
+        if (p.wait_limit <= 0 || (++polls & 15) == 0) {
             if (tail->abort_flag) return false;
             if (clock64() - t0 > p.wait_limit) {
                 tail->abort_flag = 1;
@@ -489,7 +496,7 @@ __device__ __forceinline__ bool wait_bounded_pair(uint64_t* bar, uint32_t parity
     const long long t0 = clock64();
     int polls = 0;
     while (!ptx::mbar_try_wait(bar, parity)) {
-        if ((++polls & 63) == 0) {
+        if (p.wait_limit <= 0 || (++polls & 63) == 0) {      // a zero limit gives up at the first unsuccessful poll
             if (tail->abort_flag) return false;
             if (clock64() - t0 > p.wait_limit) {
                 tail->abort_flag = 1;
@@ -895,7 +902,7 @@ __device__ __forceinline__ bool wait_bounded_d(uint64_t* bar, uint32_t parity, D
     const long long t0 = clock64();
     int polls = 0;
     while (!ptx::mbar_try_wait(bar, parity)) {
-        if ((++polls & 63) == 0) {
+        if (p.wait_limit <= 0 || (++polls & 63) == 0) {      // a zero limit gives up at the first unsuccessful poll
             if (tail->abort_flag) return false;
             if (clock64() - t0 > p.wait_limit) {
                 tail->abort_flag = 1;
@@ -975,7 +982,7 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
                     unsigned v;
                     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(dp.ready) : "memory");
                     if (v >= items_total) break;
-                    if ((++polls & 15) == 0) {
+                    if (p.wait_limit <= 0 || (++polls & 15) == 0) {
                         if (tail->abort_flag) { ok = false; break; }
                         if (clock64() - t0 > p.wait_limit) {
                             tail->abort_flag = 1;
@@ -1299,6 +1306,19 @@ bool make_tmap_out(CUtensorMap* m, const void* base, long long T, long long N, i
 static __device__ unsigned g_a_ready[kReadySlots][kMaxRowBlocks];
 static __device__ unsigned g_a_done[kReadySlots];
 
+}  // namespace
+
+void linear_reset_counters(cudaStream_t st) {
+    void *r = nullptr, *d = nullptr;
+    if (cudaGetSymbolAddress(&r, g_a_ready) == cudaSuccess && cudaGetSymbolAddress(&d, g_a_done) == cudaSuccess) {
+        cudaMemsetAsync(r, 0, sizeof(unsigned) * kReadySlots * kMaxRowBlocks, st);
+        cudaMemsetAsync(d, 0, sizeof(unsigned) * kReadySlots, st);
+        cudaStreamSynchronize(st);
+    }
+}
+
+namespace {
+
 bool next_ready_slot(unsigned** ready, unsigned** done) {
     static unsigned* ready_base[64] = {nullptr};
     static unsigned* done_base[64] = {nullptr};
@@ -1439,6 +1459,11 @@ bool single_kernel_ready(bool bf) {
 
 extern "C" {
 
+long long sasq_debug_set_wait_limit(long long cycles) {
+    const long long want = cycles < 0 ? sasq::kWaitLimit : cycles;
+    return sasq::g_wait_limit.exchange(want, std::memory_order_relaxed);
+}
+
 int sasq_static_w8a8_linear_tiles(int64_t T, int64_t N, int num_pairs, int pair_id, int32_t* tiles_host, int cap) {
     using namespace sasq;
     if (T <= 0 || N <= 0 || T > (1 << 24) || N > (1 << 24) || num_pairs <= 0 || pair_id < 0 || pair_id >= num_pairs ||
@@ -1556,7 +1581,7 @@ int linear_impl(const void* x, const int8_t* w, const float* w_scale, const floa
     p.T = (int)T; p.N = (int)N; p.K = (int)K;
     p.k_blocks = k_blocks;
     p.status = status;
-    p.wait_limit = kWaitLimit;
+    p.wait_limit = g_wait_limit.load(std::memory_order_relaxed);
     CUtensorMap tmap_a, tmap_w;
     cudaError_t e;
     if (split > 0) {
