@@ -108,8 +108,6 @@ template <int N>
 __device__ __forceinline__ void bulk_wait_group_read() {
     asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
 }
-// every bulk group of this thread has completed (writes performed)
-__device__ __forceinline__ void bulk_wait_group_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 // ---- TMEM -----------------------------------------------------------------
 // whole-warp calls (.sync.aligned)

@@ -826,7 +826,9 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive_cluster(ptx::mapa_u32(ptx::smem_u32(&tail->tmem_empty[buf]), 0));
         }
-        if (lane == 0) ptx::bulk_wait_group_all();      // output stores have left shared memory and are performed
+        // the output stores have read their shared-memory source; the writes themselves are complete by the end of
+        // the grid, which is all that a later kernel or the host can observe
+        if (lane == 0) ptx::bulk_wait_group_read<0>();
     }
 
     // ---------------- teardown ----------------

@@ -136,6 +136,15 @@ def test_llama7b_shapes_sampled_rows(T):
         check(xb, tag, w_int, w_scale, s, rows=rows)
 
 
+def test_more_channel_tiles_than_sms_takes_the_general_small_t_kernel():
+    """T <= 128 with more 128-channel tiles than the chip has SMs (N = 19200 > 148 x 128): the clustered small-T
+    kernel does not apply (its in-kernel quantizer needs every CTA resident), the 128 x 256-tile kernel with the
+    quantizer as a launch of its own does."""
+    tag, T, N, K = oracle.BF16, 24, 19200, 80
+    xb, w_int, w_scale, s = make_case(T, N, K, tag, 7400)
+    check(xb, tag, w_int, w_scale, s)
+
+
 def test_output_is_deterministic():
     tag, T, N, K = oracle.BF16, 256, 512, 1024
     xb, w_int, w_scale, s = make_case(T, N, K, tag, 7300)
