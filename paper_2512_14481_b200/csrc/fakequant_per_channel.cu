@@ -19,9 +19,16 @@ int* per_channel_status_ptr();      // the fake-quant status word (fakequant.cu)
 
 namespace {
 
+#ifndef SASQ_PC_UNROLL
+#define SASQ_PC_UNROLL 4
+#endif
+#ifndef SASQ_PC_BLOCKS_PER_SM
+#define SASQ_PC_BLOCKS_PER_SM 2
+#endif
 constexpr int kPcThreads = 256;
-constexpr int kPcUnroll = 4;            // rows in flight per thread
-constexpr int kPcMaxRowGroups = 296;    // 2 blocks per SM on 148 SMs when K fits one block column
+constexpr int kPcUnroll = SASQ_PC_UNROLL;                 // rows in flight per thread (twice as many without a backward part)
+constexpr int kPcBlocksPerSM = SASQ_PC_BLOCKS_PER_SM;
+constexpr int kPcMaxRowGroups = 148 * 4;                  // sizes the workspace
 
 struct PcParams {
     const uint4* x;
@@ -48,7 +55,7 @@ __device__ __forceinline__ void pc_store(uint4* p, const uint4& v) {
 }
 
 template <bool BF, bool FWD, bool BWD>
-__global__ void __launch_bounds__(kPcThreads, 2) fakequant_pc_kernel(const __grid_constant__ PcParams p) {
+__global__ void __launch_bounds__(kPcThreads, kPcBlocksPerSM) fakequant_pc_kernel(const __grid_constant__ PcParams p) {
     pdl_launch_dependents();
     pdl_wait();
     const int cv = blockIdx.x * blockDim.x + threadIdx.x;        // which 8-channel vector of a row
@@ -70,11 +77,12 @@ __global__ void __launch_bounds__(kPcThreads, 2) fakequant_pc_kernel(const __gri
         if (rg == 0 && bad) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
     }
     double acc[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
+    constexpr int UNROLL = BWD ? kPcUnroll : 2 * kPcUnroll;
 
-    for (long long r0 = rg; r0 < p.T; r0 += (long long)n_rg * kPcUnroll) {
-        uint4 xv[kPcUnroll], gv[kPcUnroll];
+    for (long long r0 = rg; r0 < p.T; r0 += (long long)n_rg * UNROLL) {
+        uint4 xv[UNROLL], gv[UNROLL];
 #pragma unroll
-        for (int u = 0; u < kPcUnroll; ++u) {
+        for (int u = 0; u < UNROLL; ++u) {
             const long long r = r0 + (long long)u * n_rg;
             if (r < p.T) {
                 xv[u] = pc_load(p.x + r * p.vec_per_row + cv);
@@ -82,7 +90,7 @@ __global__ void __launch_bounds__(kPcThreads, 2) fakequant_pc_kernel(const __gri
             }
         }
 #pragma unroll
-        for (int u = 0; u < kPcUnroll; ++u) {
+        for (int u = 0; u < UNROLL; ++u) {
             const long long r = r0 + (long long)u * n_rg;
             if (r < p.T) {
                 const uint32_t xw[4] = {xv[u].x, xv[u].y, xv[u].z, xv[u].w};
@@ -159,7 +167,8 @@ int pc_block_threads(int K) {
 
 int pc_row_groups(long long T, int K, int sm_count) {
     const int col_blocks = (K / 8 + kPcThreads - 1) / kPcThreads;
-    long long rg = (2LL * sm_count + col_blocks - 1) / col_blocks;       // two blocks per SM in total
+    // as many row groups as keep the whole grid resident at once (a few blocks too many would run as a second wave)
+    long long rg = ((long long)kPcBlocksPerSM * sm_count) / col_blocks;
     if (rg > kPcMaxRowGroups) rg = kPcMaxRowGroups;
     if (rg > T) rg = T;
     if (rg < 1) rg = 1;
