@@ -183,6 +183,29 @@ SASQ_API int sasq_fakequant_fwd_bwd_per_channel(const void* x, const void* grad_
                                                 const float* scales_dev, int bits, void* workspace, size_t ws_bytes,
                                                 void* stream);
 
+/* One tensor of a multi-tensor per-channel launch (host struct); fields as the arguments of
+ * sasq_fakequant_fwd_bwd_per_channel.  All descriptors of a call have the same parts (forward and / or backward). */
+typedef struct {
+    const void* x;          /* [T, K] */
+    const void* grad_y;     /* [T, K] or NULL */
+    void* y;                /* [T, K] or NULL */
+    void* grad_x;           /* [T, K] or NULL (non-NULL iff grad_y is) */
+    const float* scales;    /* [K] fp32, device */
+    float* grad_scales;     /* [K] fp32, device (needed with a backward part) */
+    int64_t T, K;
+    int64_t reserved;       /* must be 0 */
+} sasq_pcdesc_t;
+
+/* Bytes of scratch for a multi-tensor per-channel call whose tensors have total_K channels in all. */
+SASQ_API size_t sasq_fakequant_per_channel_multi_workspace(int64_t total_K);
+
+/* Up to 16 per-channel quantizers in one launch (e.g. the seven linear inputs of a decoder layer): the tensors run
+ * side by side, each on a share of the GPU in proportion to its size.  descs_host: HOST array, copied into the launch
+ * parameters.  Results are those of n_tensors separate calls. */
+SASQ_API int sasq_fakequant_fwd_bwd_per_channel_multi(const sasq_pcdesc_t* descs_host, int n_tensors, int accumulate,
+                                                      int dt, int bits, void* workspace, size_t ws_bytes,
+                                                      void* stream);
+
 /* Bytes of scratch sasq_static_w8a8_linear needs for this shape (may be 0). */
 SASQ_API size_t sasq_static_w8a8_linear_workspace(int64_t T, int64_t N, int64_t K);
 

@@ -21,7 +21,8 @@ __all__ = [
     "sasq_quantize_weight", "linear_launches", "sasq_fakequant_fwd_bwd_static", "sasq_static_w8a8_linear_tiles",
     "sasq_fakequant_per_channel_workspace", "sasq_fakequant_fwd_bwd_per_channel",
     "sasq_fakequant_fwd_bwd_ablation", "sasq_adamw_scales", "SASQ_FULL_OPERATOR", "SASQ_WITHOUT_ROUND",
-    "SASQ_WITHOUT_CLAMP", "sasq_dynamic_w8a8_linear_workspace", "sasq_dynamic_w8a8_linear", "sasq_debug_set_wait_limit",
+    "SASQ_WITHOUT_CLAMP", "sasq_dynamic_w8a8_linear_workspace", "sasq_dynamic_w8a8_linear", "sasq_debug_set_wait_limit", "PcDesc", "sasq_fakequant_per_channel_multi_workspace",
+    "sasq_fakequant_fwd_bwd_per_channel_multi",
 ]
 
 SASQ_F16 = 0
@@ -54,6 +55,13 @@ class QDesc(ctypes.Structure):
     _fields_ = [("x", ctypes.c_void_p), ("grad_y", ctypes.c_void_p), ("y", ctypes.c_void_p),
                 ("grad_x", ctypes.c_void_p), ("numel", ctypes.c_int64), ("scale_index", ctypes.c_int32),
                 ("reserved", ctypes.c_int32)]
+
+
+class PcDesc(ctypes.Structure):
+    """Mirror of sasq_pcdesc_t."""
+    _fields_ = [("x", ctypes.c_void_p), ("grad_y", ctypes.c_void_p), ("y", ctypes.c_void_p),
+                ("grad_x", ctypes.c_void_p), ("scales", ctypes.c_void_p), ("grad_scales", ctypes.c_void_p),
+                ("T", ctypes.c_int64), ("K", ctypes.c_int64), ("reserved", ctypes.c_int64)]
 
 
 def library_path() -> str:
@@ -103,6 +111,10 @@ def load_library() -> ctypes.CDLL:
     L.sasq_dynamic_w8a8_linear_workspace.argtypes = [i64, i64, i64]
     L.sasq_dynamic_w8a8_linear.restype = i32
     L.sasq_dynamic_w8a8_linear.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, sz, vp]
+    L.sasq_fakequant_per_channel_multi_workspace.restype = sz
+    L.sasq_fakequant_per_channel_multi_workspace.argtypes = [i64]
+    L.sasq_fakequant_fwd_bwd_per_channel_multi.restype = i32
+    L.sasq_fakequant_fwd_bwd_per_channel_multi.argtypes = [ctypes.POINTER(PcDesc), i32, i32, i32, i32, vp, sz, vp]
     L.sasq_debug_set_wait_limit.restype = ctypes.c_longlong
     L.sasq_debug_set_wait_limit.argtypes = [ctypes.c_longlong]
     L.sasq_static_w8a8_linear_tiles.restype = i32
@@ -287,6 +299,41 @@ def sasq_fakequant_fwd_bwd_per_channel(x, grad_y, y, grad_x, grad_scales, scales
                                                              x.shape[1], _dt(x), _ptr(scales), int(bits),
                                                              _ptr(workspace), _nbytes(workspace), _stream(stream)),
            "sasq_fakequant_fwd_bwd_per_channel")
+
+
+def sasq_fakequant_per_channel_multi_workspace(total_K: int) -> int:
+    return int(load_library().sasq_fakequant_per_channel_multi_workspace(int(total_K)))
+
+
+def sasq_fakequant_fwd_bwd_per_channel_multi(tensors, workspace, bits: int = 8, accumulate: bool = False,
+                                             stream=None) -> None:
+    """tensors: sequence of (x [T, K], grad_y | None, y | None, grad_x | None, scales [K], grad_scales [K] | None)."""
+    n = len(tensors)
+    descs = (PcDesc * max(n, 1))()
+    dt = None
+    for i, (x, gy, y, gx, sc, gs) in enumerate(tensors):
+        _dev(x, "x"); _dev(sc, "scales", torch.float32)
+        if x.dim() != 2 or sc.numel() != x.shape[1]:
+            raise ValueError("x must be [T, K] and scales [K]")
+        for name, t in (("grad_y", gy), ("y", y), ("grad_x", gx)):
+            if t is not None:
+                _dev(t, name, x.dtype)
+                if tuple(t.shape) != tuple(x.shape):
+                    raise ValueError(f"{name} must have the shape of x")
+        if gs is not None:
+            _dev(gs, "grad_scales", torch.float32)
+        if dt is None:
+            dt = _dt(x)
+        elif dt != _dt(x):
+            raise TypeError("all tensors of one call must share a dtype")
+        descs[i] = PcDesc(_ptr(x), _ptr(gy), _ptr(y), _ptr(gx), _ptr(sc), _ptr(gs), x.shape[0], x.shape[1], 0)
+    if workspace is not None:
+        _dev(workspace, "workspace")
+    _check(load_library().sasq_fakequant_fwd_bwd_per_channel_multi(descs, n, int(bool(accumulate)),
+                                                                   SASQ_BF16 if dt is None else dt, int(bits),
+                                                                   _ptr(workspace), _nbytes(workspace),
+                                                                   _stream(stream)),
+           "sasq_fakequant_fwd_bwd_per_channel_multi")
 
 
 def sasq_static_w8a8_linear_workspace(T: int, N: int, K: int) -> int:

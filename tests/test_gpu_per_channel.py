@@ -124,3 +124,31 @@ def test_errors_and_edge_cases():
     sc.fill_(1.0)
     P.sasq_fakequant_fwd_bwd_per_channel(e0, e0, e0, e0, grads, sc, ws, 8)
     assert float(grads.abs().sum()) == 0.0
+
+
+def test_multi_tensor_launch_matches_the_oracle_per_tensor():
+    """The seven linear inputs of a (scaled-down) decoder layer in one launch, plus an empty tensor."""
+    tag, bits = oracle.BF16, 8
+    shapes = [(67, 512)] * 3 + [(67, 1376), (5, 264), (0, 16), (300, 2056)]
+    cases = [make(max(T, 1), K, tag, 9300 + i) for i, (T, K) in enumerate(shapes)]
+    tensors, keep = [], []
+    total_k = sum(K for _, K in shapes)
+    for (T, K), (xb, gb, s) in zip(shapes, cases):
+        xb, gb = xb[:T], gb[:T]
+        x = oracle.tensor_of(xb, tag).cuda().reshape(T, K)
+        g = oracle.tensor_of(gb, tag).cuda().reshape(T, K)
+        y, dx = torch.empty_like(x), torch.empty_like(x)
+        sc, gs = torch.from_numpy(s).cuda(), torch.full((K,), 3.0, device="cuda")
+        tensors.append((x, g, y, dx, sc, gs))
+        keep.append((xb, gb, s))
+    ws = torch.empty(P.sasq_fakequant_per_channel_multi_workspace(total_k), dtype=torch.uint8, device="cuda")
+    P.sasq_fakequant_fwd_bwd_per_channel_multi(tensors, ws, bits)
+    assert P.sasq_device_status() == 0
+    for (T, K), (x, g, y, dx, sc, gs), (xb, gb, s) in zip(shapes, tensors, keep):
+        if T == 0:
+            assert float(gs.abs().sum()) == 0.0
+            continue
+        y_o, _ = oracle.fakequant_fwd_per_channel(xb, tag, s, bits)
+        dx_o, ds_o = oracle.fakequant_bwd_per_channel(xb, gb, tag, s, bits)
+        assert np.array_equal(host_bits(y), y_o) and np.array_equal(host_bits(dx), dx_o)
+        check_ds(gs.cpu().numpy(), ds_o, gb, tag, bits)
