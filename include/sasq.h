@@ -224,6 +224,23 @@ SASQ_API int sasq_static_w8a8_linear(const void* x, const int8_t* w, const float
                             const void* bias, void* y, int32_t* acc_out, int64_t T, int64_t N, int64_t K,
                             int dt, int bits, void* workspace, size_t ws_bytes, void* stream);
 
+/* Bytes of scratch sasq_static_w8a8_linear_per_channel needs for this shape. */
+SASQ_API size_t sasq_static_w8a8_linear_per_channel_workspace(int64_t T, int64_t N, int64_t K);
+
+/* Static W8A8 linear with one learned activation factor per CHANNEL (column of x), the granularity of the paper's
+ * experiments (Sec. 5.1).  Because the factors are static, they are absorbed into the frozen weights ahead of time
+ * instead of being carried through Eq. 3's groups: the caller quantizes w'[n,k] = w_fp[n,k] * s_x[k] per output
+ * channel (sasq_quantize_weight) and passes the result as w, w_scale.  The call then computes
+ *   X_int[t,k] = int8(c(x[t,k])) with s = x_scales_dev[k]        (Eq. 1 per channel, no run-time scale pass)
+ *   acc[t,n]   = sum_k X_int[t,k] * w[n,k]                        (= sum_k X_int s_x[k] w_fp[n,k] / w_scale[n], up to the
+ *                                                                  weight rounding)
+ *   y[t,n]     = narrow( fl32(acc) * w_scale[n] (+ bias[n]) )
+ * x_scales_dev: [K] fp32.  Other arguments as for sasq_static_w8a8_linear. */
+SASQ_API int sasq_static_w8a8_linear_per_channel(const void* x, const int8_t* w, const float* w_scale,
+                                                 const float* x_scales_dev, const void* bias, void* y,
+                                                 int32_t* acc_out, int64_t T, int64_t N, int64_t K, int dt, int bits,
+                                                 void* workspace, size_t ws_bytes, void* stream);
+
 /* Bytes of scratch sasq_dynamic_w8a8_linear needs for this shape. */
 SASQ_API size_t sasq_dynamic_w8a8_linear_workspace(int64_t T, int64_t N, int64_t K);
 

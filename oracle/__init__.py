@@ -296,3 +296,15 @@ def w8a8_linear_dynamic(x: np.ndarray, tag: int, w_int: np.ndarray, w_scale: np.
         y_t, _, acc_t = w8a8_linear(row, tag, w_int, w_scale, float(s), bits, bias)
         y[t], acc[t] = y_t[0], acc_t[0]
     return y, acc, s_rows
+
+
+def w8a8_linear_per_channel(x: np.ndarray, tag: int, w_int: np.ndarray, w_scale: np.ndarray, s_vec: np.ndarray,
+                            bits: int = 8, bias: np.ndarray | None = None):
+    """Static W8A8 linear with one activation factor per channel whose values were folded into the weights ahead of
+    time (w_int, w_scale quantize w_fp[n,k] * s_vec[k]): Eq. 1 per channel, the integer GEMM, then Eq. 2 with the
+    activation factor already inside the weights (output factor w_scale[n] alone).  Built from the pinned pieces.
+    Returns (y bits, acc int32)."""
+    _, codes = fakequant_fwd_per_channel(x, tag, s_vec, bits)
+    acc = int_gemm(codes.astype(np.int8), w_int)
+    y, _ = dequant(acc, w_scale, 1.0, tag, bias)
+    return y, acc

@@ -22,7 +22,8 @@ __all__ = [
     "sasq_fakequant_per_channel_workspace", "sasq_fakequant_fwd_bwd_per_channel",
     "sasq_fakequant_fwd_bwd_ablation", "sasq_adamw_scales", "SASQ_FULL_OPERATOR", "SASQ_WITHOUT_ROUND",
     "SASQ_WITHOUT_CLAMP", "sasq_dynamic_w8a8_linear_workspace", "sasq_dynamic_w8a8_linear", "sasq_debug_set_wait_limit", "PcDesc", "sasq_fakequant_per_channel_multi_workspace",
-    "sasq_fakequant_fwd_bwd_per_channel_multi",
+    "sasq_fakequant_fwd_bwd_per_channel_multi", "sasq_static_w8a8_linear_per_channel_workspace",
+    "sasq_static_w8a8_linear_per_channel",
 ]
 
 SASQ_F16 = 0
@@ -107,6 +108,10 @@ def load_library() -> ctypes.CDLL:
     L.sasq_fakequant_per_channel_workspace.argtypes = [i64, i64]
     L.sasq_fakequant_fwd_bwd_per_channel.restype = i32
     L.sasq_fakequant_fwd_bwd_per_channel.argtypes = [vp, vp, vp, vp, vp, i32, i64, i64, i32, vp, i32, vp, sz, vp]
+    L.sasq_static_w8a8_linear_per_channel_workspace.restype = sz
+    L.sasq_static_w8a8_linear_per_channel_workspace.argtypes = [i64, i64, i64]
+    L.sasq_static_w8a8_linear_per_channel.restype = i32
+    L.sasq_static_w8a8_linear_per_channel.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, sz, vp]
     L.sasq_dynamic_w8a8_linear_workspace.restype = sz
     L.sasq_dynamic_w8a8_linear_workspace.argtypes = [i64, i64, i64]
     L.sasq_dynamic_w8a8_linear.restype = i32
@@ -362,6 +367,33 @@ def sasq_static_w8a8_linear(x, w, w_scale, x_scale, y, bias=None, acc_out=None, 
     _check(load_library().sasq_static_w8a8_linear(_ptr(x), _ptr(w), _ptr(w_scale), _ptr(x_scale), _ptr(bias), _ptr(y),
                                                   _ptr(acc_out), T, N, K, _dt(x), int(bits), _ptr(workspace),
                                                   _nbytes(workspace), _stream(stream)), "sasq_static_w8a8_linear")
+
+
+def sasq_static_w8a8_linear_per_channel_workspace(T: int, N: int, K: int) -> int:
+    return int(load_library().sasq_static_w8a8_linear_per_channel_workspace(int(T), int(N), int(K)))
+
+
+def sasq_static_w8a8_linear_per_channel(x, w, w_scale, x_scales, y, bias=None, acc_out=None, workspace=None,
+                                        bits: int = 8, stream=None) -> None:
+    """x [T, K], x_scales [K] (one static factor per channel, already folded into w), w [N, K] int8, y [T, N]."""
+    _dev(x, "x"); _dev(w, "w", torch.int8); _dev(w_scale, "w_scale", torch.float32)
+    _dev(x_scales, "x_scales", torch.float32); _dev(y, "y", x.dtype)
+    for name, t, dtp in (("bias", bias, x.dtype), ("acc_out", acc_out, torch.int32)):
+        if t is not None:
+            _dev(t, name, dtp)
+    if workspace is not None:
+        _dev(workspace, "workspace")
+    if x.dim() != 2 or w.dim() != 2 or x.shape[1] != w.shape[1] or x_scales.numel() != x.shape[1]:
+        raise ValueError("x must be [T, K], w [N, K] and x_scales [K]")
+    T, K = x.shape
+    N = w.shape[0]
+    if tuple(y.shape) != (T, N) or w_scale.numel() != N or (bias is not None and bias.numel() != N):
+        raise ValueError("y must be [T, N], w_scale and bias [N]")
+    _check(load_library().sasq_static_w8a8_linear_per_channel(_ptr(x), _ptr(w), _ptr(w_scale), _ptr(x_scales),
+                                                              _ptr(bias), _ptr(y), _ptr(acc_out), T, N, K, _dt(x),
+                                                              int(bits), _ptr(workspace), _nbytes(workspace),
+                                                              _stream(stream)),
+           "sasq_static_w8a8_linear_per_channel")
 
 
 def sasq_dynamic_w8a8_linear_workspace(T: int, N: int, K: int) -> int:

@@ -64,6 +64,8 @@ struct LinearParams {
     const float* w_scale;
     const float* x_scale;      // one static factor for the whole tensor, or
     const float* row_scale;    // [T] one factor per row (dynamic per-token quantization); then x_scale is unused
+    const float* chan_inv;     // [K] fl32(1 / s_x[k]) for one static factor per channel; the output factor is then
+                               // w_scale[n] alone (the caller folded s_x[k] into the weights); x_scale is unused
     const void* bias;
     void* y;
     int32_t* acc_out;
@@ -224,8 +226,9 @@ w8a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         const int quad = warp & 3;                      // TMEM lane quadrant this warp may read
         const int et = threadIdx.x - 64;                // 0..127
         const bool per_row = p.row_scale != nullptr;
-        const float sx = per_row ? 1.0f : __ldg(p.x_scale);
-        if (!per_row && blockIdx.x == 0 && et == 0 && scale_is_bad(sx)) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
+        const bool one_factor = !per_row && p.chan_inv == nullptr;       // one static factor for the whole tensor
+        const float sx = one_factor ? __ldg(p.x_scale) : 1.0f;
+        if (one_factor && blockIdx.x == 0 && et == 0 && scale_is_bad(sx)) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
         bool ok = true;
         int it = 0;
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
@@ -407,6 +410,28 @@ __device__ __forceinline__ uint2 quantize8(const uint4& v, float inv, float qn, 
     return make_uint2(lo, hi);
 }
 
+// the same with one factor per channel: inv8 points at the reciprocals of the 8 channels of this word
+template <bool BF>
+__device__ __forceinline__ uint2 quantize8_channels(const uint4& v, const float* inv8, float qn, float qp) {
+    const float4 ia = __ldg(reinterpret_cast<const float4*>(inv8));
+    const float4 ib = __ldg(reinterpret_cast<const float4*>(inv8) + 1);
+    const float inv[8] = {ia.x, ia.y, ia.z, ia.w, ib.x, ib.y, ib.z, ib.w};
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    int c[8];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const float2 f = widen2<BF>(w[q]);
+        c[2 * q] = __float2int_rn(fminf(fmaxf(__fmul_rn(f.x, inv[2 * q]), -qn), qp));
+        c[2 * q + 1] = __float2int_rn(fminf(fmaxf(__fmul_rn(f.y, inv[2 * q + 1]), -qn), qp));
+    }
+    uint32_t lo, hi, t;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(t) : "r"(c[3]), "r"(c[2]), "r"(0));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(lo) : "r"(c[1]), "r"(c[0]), "r"(t));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(t) : "r"(c[7]), "r"(c[6]), "r"(0));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(c[5]), "r"(c[4]), "r"(t));
+    return make_uint2(lo, hi);
+}
+
 __device__ __forceinline__ uint4 ld_stream16(const uint4* p) {
     uint4 v;
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
@@ -423,6 +448,8 @@ struct ConvJob {
     long long items_per_block;   // items per 256-row block
     float inv, qn, qp;
     bool eight;
+    const float* chan_inv;       // per-channel reciprocals, or NULL
+    unsigned vec_per_row;        // K / 8
 };
 
 __device__ __forceinline__ void conv_load(const ConvJob& j, long long c, int lane, uint4 (&v)[CONV_ITEMS]) {
@@ -435,7 +462,14 @@ __device__ __forceinline__ void conv_load(const ConvJob& j, long long c, int lan
 
 template <bool BF>
 __device__ __forceinline__ void conv_store(const ConvJob& j, long long c, int lane, const uint4 (&v)[CONV_ITEMS]) {
-    if (j.eight) {
+    if (j.chan_inv != nullptr) {
+#pragma unroll
+        for (int u = 0; u < CONV_ITEMS; ++u) {
+            const long long i = c * CONV_CHUNK + u * 32 + lane;
+            if (i < j.total)
+                j.dst[i] = quantize8_channels<BF>(v[u], j.chan_inv + 8 * (unsigned)(i % j.vec_per_row), j.qn, j.qp);
+        }
+    } else if (j.eight) {
 #pragma unroll
         for (int u = 0; u < CONV_ITEMS; ++u) {
             const long long i = c * CONV_CHUNK + u * 32 + lane;
@@ -566,7 +600,9 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         job.ready = pp.ready;
         job.total = (long long)p.T * (p.K >> 3);
         job.items_per_block = (long long)PBM * (p.K >> 3);
-        job.inv = __fdiv_rn(1.0f, __ldg(p.x_scale));
+        job.chan_inv = p.chan_inv;
+        job.vec_per_row = (unsigned)(p.K >> 3);
+        job.inv = p.chan_inv == nullptr ? __fdiv_rn(1.0f, __ldg(p.x_scale)) : 0.0f;
         job.qn = pp.qn;
         job.qp = pp.qp;
         job.eight = pp.qp == 127.0f;
@@ -699,8 +735,9 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         const int quad = warp & 3;
         const int et = threadIdx.x - 64;
         const bool per_row = p.row_scale != nullptr;
-        const float sx = per_row ? 1.0f : __ldg(p.x_scale);
-        if (!per_row && blockIdx.x == 0 && et == 0 && scale_is_bad(sx)) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
+        const bool one_factor = !per_row && p.chan_inv == nullptr;       // one static factor for the whole tensor
+        const float sx = one_factor ? __ldg(p.x_scale) : 1.0f;
+        if (one_factor && blockIdx.x == 0 && et == 0 && scale_is_bad(sx)) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
         const bool has_bias = p.bias != nullptr;
         bool ok = true;
         int it = 0;
@@ -1046,8 +1083,9 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
         // ---------------- activation quantizer, then epilogue (warps 2..5) ----------------
         const int et = threadIdx.x - 64;                       // 0..127
         const bool per_row = p.row_scale != nullptr;
-        const float sx = per_row ? 1.0f : __ldg(p.x_scale);
-        if (!per_row && blockIdx.x == 0 && et == 0 && scale_is_bad(sx)) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
+        const bool one_factor = !per_row && p.chan_inv == nullptr;       // one static factor for the whole tensor
+        const float sx = one_factor ? __ldg(p.x_scale) : 1.0f;
+        if (one_factor && blockIdx.x == 0 && et == 0 && scale_is_bad(sx)) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
         if (dp.x != nullptr) {
             const float inv = __fdiv_rn(1.0f, sx);
             const uint4* src = reinterpret_cast<const uint4*>(dp.x);
@@ -1055,8 +1093,15 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
             unsigned mine = 0;
             for (unsigned i = blockIdx.x * 128u + (unsigned)et; i < items_total; i += gridDim.x * 128u) {
                 const uint4 a = ld_stream16(src + 2 * (size_t)i), b = ld_stream16(src + 2 * (size_t)i + 1);
-                const uint2 lo = quantize8<BF, false>(a, inv, dp.qn, dp.qp);
-                const uint2 hi = quantize8<BF, false>(b, inv, dp.qn, dp.qp);
+                uint2 lo, hi;
+                if (p.chan_inv != nullptr) {
+                    const float* ci = p.chan_inv + 16 * (i % (unsigned)(p.K >> 4));
+                    lo = quantize8_channels<BF>(a, ci, dp.qn, dp.qp);
+                    hi = quantize8_channels<BF>(b, ci + 8, dp.qn, dp.qp);
+                } else {
+                    lo = quantize8<BF, false>(a, inv, dp.qn, dp.qp);
+                    hi = quantize8<BF, false>(b, inv, dp.qn, dp.qp);
+                }
                 dst[i] = make_uint4(lo.x, lo.y, hi.x, hi.y);
                 ++mine;
             }
@@ -1120,7 +1165,7 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
         const int pstride = dp.tp + 4;
         const bool has_bias = p.bias != nullptr;
         const bool per_row = p.row_scale != nullptr;
-        const float sx = per_row ? 1.0f : __ldg(p.x_scale);
+        const float sx = (per_row || p.chan_inv != nullptr) ? 1.0f : __ldg(p.x_scale);
         const int items = rows * (dp.tp >> 2);
         const int32_t* slots = reinterpret_cast<const int32_t*>(ring + dp.slots_offset);
         for (int it = et; it < items; it += 128) {
@@ -1172,11 +1217,26 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
 template <bool BF>
 __global__ void __launch_bounds__(256) quantize_act_kernel(const uint4* __restrict__ x, uint2* __restrict__ out,
                                                            long long n8, const float* __restrict__ x_scale,
+                                                           const float* __restrict__ chan_inv, unsigned vec_per_row,
                                                            float qn, float qp) {
-    const float inv = __fdiv_rn(1.0f, __ldg(x_scale));
+    pdl_wait();
+    const float inv = chan_inv == nullptr ? __fdiv_rn(1.0f, __ldg(x_scale)) : 0.0f;
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += stride)
-        out[i] = quantize8<BF, false>(x[i], inv, qn, qp);
+        out[i] = chan_inv == nullptr ? quantize8<BF, false>(x[i], inv, qn, qp)
+                                     : quantize8_channels<BF>(x[i], chan_inv + 8 * (unsigned)(i % vec_per_row), qn, qp);
+}
+
+// reciprocals of the per-channel factors, fl32(1 / s[k]), once per call; a zero / non-finite factor is reported
+__global__ void __launch_bounds__(256) reciprocal_factors_kernel(const float* __restrict__ s, float* __restrict__ inv,
+                                                                 int K, int* status) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int k = blockIdx.x * 256 + threadIdx.x;
+    if (k >= K) return;
+    const float sk = s[k];
+    if (scale_is_bad(sk)) atomicMax(status, (int)SASQ_ERR_BAD_SCALE);
+    inv[k] = __fdiv_rn(1.0f, sk);
 }
 
 // Dynamic per-token quantization (Sec. 4.4, generation phase): one block per row of x.  The row's factor is its
@@ -1500,13 +1560,15 @@ namespace {
 
 // dynamic == false: static factor x_scale_dev (the hot path).  dynamic == true: every row gets its own max-based
 // factor, written to row_scale_out (or to the workspace when that is NULL) by a launch that also quantizes the rows.
-int linear_impl(const void* x, const int8_t* w, const float* w_scale, const float* x_scale_dev, bool dynamic,
-                float* row_scale_out, const void* bias, void* y, int32_t* acc_out, int64_t T, int64_t N, int64_t K,
+int linear_impl(const void* x, const int8_t* w, const float* w_scale, const float* x_scale_dev,
+                const float* x_scales_vec, bool dynamic, float* row_scale_out, const void* bias, void* y, int32_t* acc_out, int64_t T, int64_t N, int64_t K,
                 int dt, int bits, void* workspace, size_t ws_bytes, void* stream) {
     if (T < 0 || N <= 0 || K <= 0) return SASQ_ERR_INVALID_ARG;
     if (dt != SASQ_F16 && dt != SASQ_BF16) return SASQ_ERR_INVALID_ARG;
     if (bits < 2 || bits > 8) return SASQ_ERR_INVALID_ARG;
-    if (w == nullptr || w_scale == nullptr || (!dynamic && x_scale_dev == nullptr)) return SASQ_ERR_INVALID_ARG;
+    if (w == nullptr || w_scale == nullptr || (!dynamic && x_scale_dev == nullptr && x_scales_vec == nullptr))
+        return SASQ_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(x_scales_vec) & 3u) return SASQ_ERR_INVALID_ARG;
     if (T > 0 && (x == nullptr || y == nullptr)) return SASQ_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(row_scale_out) & 3u) return SASQ_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(acc_out) ||
@@ -1515,7 +1577,8 @@ int linear_impl(const void* x, const int8_t* w, const float* w_scale, const floa
     if (K % 16 != 0 || N % 8 != 0 || K > 131072 || T > (1 << 24) || N > (1 << 24)) return SASQ_ERR_UNSUPPORTED;
     if (T == 0) return SASQ_OK;
     const size_t ws_need = dynamic ? sasq_dynamic_w8a8_linear_workspace(T, N, K)
-                                   : sasq_static_w8a8_linear_workspace(T, N, K);
+                           : x_scales_vec != nullptr ? sasq_static_w8a8_linear_per_channel_workspace(T, N, K)
+                                                     : sasq_static_w8a8_linear_workspace(T, N, K);
     if (workspace == nullptr || !aligned16(workspace) || ws_bytes < ws_need) return SASQ_ERR_WORKSPACE;
     const int sm_count = device_sm_count_if_sm100();
     if (sm_count <= 0) return SASQ_ERR_UNSUPPORTED;
@@ -1534,6 +1597,21 @@ int linear_impl(const void* x, const int8_t* w, const float* w_scale, const floa
                           ? decode_split(dt == SASQ_BF16, n_tiles128, k_blocks, sm_count, kDecodeSmem) : 0;
     const bool in_kernel_quantizer = !dynamic && (split > 0 || (T > BM && (T + PBM - 1) / PBM <= kMaxRowBlocks));
     const float* row_scale = nullptr;
+    const float* chan_inv = nullptr;
+    if (x_scales_vec != nullptr) {
+        // one static factor per channel: their reciprocals go to the workspace (behind the codes) once per call
+        float* inv = reinterpret_cast<float*>(reinterpret_cast<uintptr_t>(a_int8) + (uintptr_t)((T * K + 255) / 256 * 256));
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((unsigned)((K + 255) / 256), 1, 1);
+        cfg.blockDim = dim3(256, 1, 1);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1] = {pdl_attribute()};
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, reciprocal_factors_kernel, x_scales_vec, inv, (int)K, status) != cudaSuccess)
+            return SASQ_ERR_CUDA;
+        chan_inv = inv;
+    }
     if (dynamic) {
         // per-token factors and codes by a launch of their own (the factor of a row needs the whole row first)
         float* rs = row_scale_out;
@@ -1564,11 +1642,11 @@ int linear_impl(const void* x, const int8_t* w, const float* w_scale, const floa
         if (dt == SASQ_BF16)
             quantize_act_kernel<true><<<(int)blocks, 256, 0, st>>>(static_cast<const uint4*>(x),
                                                                    reinterpret_cast<uint2*>(a_int8), n8,
-                                                                   x_scale_dev, qn, qp);
+                                                                   x_scale_dev, chan_inv, (unsigned)(K / 8), qn, qp);
         else
             quantize_act_kernel<false><<<(int)blocks, 256, 0, st>>>(static_cast<const uint4*>(x),
                                                                     reinterpret_cast<uint2*>(a_int8), n8,
-                                                                    x_scale_dev, qn, qp);
+                                                                    x_scale_dev, chan_inv, (unsigned)(K / 8), qn, qp);
         if (cudaGetLastError() != cudaSuccess) return SASQ_ERR_CUDA;
     }
 
@@ -1577,6 +1655,7 @@ int linear_impl(const void* x, const int8_t* w, const float* w_scale, const floa
     p.w_scale = w_scale;
     p.x_scale = x_scale_dev;
     p.row_scale = row_scale;
+    p.chan_inv = chan_inv;
     p.bias = bias;
     p.y = y;
     p.acc_out = acc_out;
@@ -1685,7 +1764,22 @@ extern "C" {
 int sasq_static_w8a8_linear(const void* x, const int8_t* w, const float* w_scale, const float* x_scale_dev,
                             const void* bias, void* y, int32_t* acc_out, int64_t T, int64_t N, int64_t K, int dt,
                             int bits, void* workspace, size_t ws_bytes, void* stream) {
-    return sasq::linear_impl(x, w, w_scale, x_scale_dev, false, nullptr, bias, y, acc_out, T, N, K, dt, bits,
+    return sasq::linear_impl(x, w, w_scale, x_scale_dev, nullptr, false, nullptr, bias, y, acc_out, T, N, K, dt, bits,
+                             workspace, ws_bytes, stream);
+}
+
+size_t sasq_static_w8a8_linear_per_channel_workspace(int64_t T, int64_t N, int64_t K) {
+    if (T <= 0 || K <= 0) return 0;
+    // int8 codes, then one fp32 reciprocal per channel
+    return sasq_static_w8a8_linear_workspace(T, N, K) + 256 + (size_t)K * sizeof(float) + 256;
+}
+
+int sasq_static_w8a8_linear_per_channel(const void* x, const int8_t* w, const float* w_scale,
+                                        const float* x_scales_dev, const void* bias, void* y, int32_t* acc_out,
+                                        int64_t T, int64_t N, int64_t K, int dt, int bits, void* workspace,
+                                        size_t ws_bytes, void* stream) {
+    if (x_scales_dev == nullptr) return SASQ_ERR_INVALID_ARG;
+    return sasq::linear_impl(x, w, w_scale, nullptr, x_scales_dev, false, nullptr, bias, y, acc_out, T, N, K, dt, bits,
                              workspace, ws_bytes, stream);
 }
 
@@ -1698,7 +1792,7 @@ size_t sasq_dynamic_w8a8_linear_workspace(int64_t T, int64_t N, int64_t K) {
 int sasq_dynamic_w8a8_linear(const void* x, const int8_t* w, const float* w_scale, const void* bias, void* y,
                              float* row_scale_out, int32_t* acc_out, int64_t T, int64_t N, int64_t K, int dt, int bits,
                              void* workspace, size_t ws_bytes, void* stream) {
-    return sasq::linear_impl(x, w, w_scale, nullptr, true, row_scale_out, bias, y, acc_out, T, N, K, dt, bits,
+    return sasq::linear_impl(x, w, w_scale, nullptr, nullptr, true, row_scale_out, bias, y, acc_out, T, N, K, dt, bits,
                              workspace, ws_bytes, stream);
 }
 
