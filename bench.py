@@ -46,7 +46,7 @@ INT8_OVER_BF16_NOMINAL = 2.0          # dense INT8 peak is twice the dense bf16 
 # DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/ (T = 2048 workload only;
 # set to None whenever the kernel changes after its capture)
 NCU_TRAFFIC_FAKEQUANT = 533.2e6        # profiles/fakequant_kernel_llama7b_layer_T2048.md
-NCU_TRAFFIC_GEMM_MEAN = 473.1e6 / 7    # profiles/w8a8_gemm_pair_kernel_T2048.md: mean over the step's seven launches
+NCU_TRAFFIC_GEMM = None                # DRAM bytes of the step's one GEMM launch (profiles/w8a8_gemm_pair_kernel_T2048.md)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -136,7 +136,7 @@ def physical_gpu_index(local_rank: int) -> int:
 # the workload on the device
 # ---------------------------------------------------------------------------
 class Layer:
-    def __init__(self, P, device, rank: int):
+    def __init__(self, P, device, rank: int, linear_calls: str = "layer"):
         self.P = P
         dt = torch.bfloat16
         self.x, self.g, self.y, self.dx, self.w_int, self.w_scale, self.out = [], [], [], [], [], [], []
@@ -162,25 +162,36 @@ class Layer:
         self.scales = scales
         self.grads = torch.zeros(7, dtype=torch.float32, device=device)
         self.q_ws = torch.empty(P.sasq_fakequant_multi_workspace(7), dtype=torch.uint8, device=device)
-        self.l_ws = torch.empty(max(P.sasq_static_w8a8_linear_workspace(T_TOKENS, N, K)
-                                    for _, K, N in W.LLAMA2_7B_LINEARS), dtype=torch.uint8, device=device)
+        self.shapes = [(T_TOKENS, N, K) for _, K, N in W.LLAMA2_7B_LINEARS]
+        self.l_ws = torch.empty(P.sasq_static_w8a8_linear_multi_workspace(self.shapes), dtype=torch.uint8,
+                                device=device)
+        self.linears = [(self.x[i], self.w_int[i], self.w_scale[i], self.scales[i:i + 1], self.out[i])
+                        for i in range(7)]
+        self.calls = LINEAR_CALLS[linear_calls]
         self.descs = [(self.x[i], self.g[i], self.y[i], self.dx[i], i) for i in range(7)]
         torch.cuda.synchronize()
         assert P.sasq_device_status() == 0
 
     # kernels launched per step: one fused quantizer launch (the reduction's second stage runs in its last block),
-    # then one launch per linear (its activation quantizer runs inside the GEMM kernel)
+    # then the linears (activation quantizer inside the GEMM kernel): the seven problems of the step are independent
+    # and resident, so by default they are submitted in one call, which runs them in one launch while their int8
+    # codes fit L2; the other groupings are there for comparison
     def phase_a(self):
         self.P.sasq_fakequant_fwd_bwd_multi(self.descs, self.scales, self.grads, self.q_ws, BITS)
         return 1
 
     def phase_b(self):
         n = 0
-        for i in range(7):
-            self.P.sasq_static_w8a8_linear(self.x[i], self.w_int[i], self.w_scale[i], self.scales[i:i + 1],
-                                           self.out[i], workspace=self.l_ws, bits=BITS)
-            n += self.P.linear_launches(T_TOKENS)
+        for call in self.calls:
+            self.P.sasq_static_w8a8_linear_multi([self.linears[i] for i in call], self.l_ws, bits=BITS)
+            n += self.P.linear_multi_launches([self.shapes[i] for i in call])
         return n
+
+
+# how phase B submits the seven linears: all in one call; the groups a decoder layer's data flow allows
+# (q/k/v, o, gate/up, down); or one call per linear
+LINEAR_CALLS = {"layer": [[0, 1, 2, 3, 4, 5, 6]], "dependent": [[0, 1, 2], [3], [4, 5], [6]],
+                "each": [[i] for i in range(7)]}
 
 
 def max_over_ranks(values, dist, device):
@@ -212,7 +223,7 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=device)
 
-    layer = Layer(P, device, rank)
+    layer = Layer(P, device, rank, args.linear_calls)
     stream = torch.cuda.current_stream()
 
     def barrier():
@@ -270,6 +281,7 @@ def run_ours(args):
         "data": "synthetic",
         "config": {"workload": WORKLOAD, "tokens": T_TOKENS, "bits": BITS, "tensors": 7,
                    "phases": "A: fused fake-quant fwd+bwd + scale-gradient reduction; B: 7 static W8A8 linears",
+                   "linear_calls": args.linear_calls,
                    "l2": f"inputs larger than L2 ({qbytes / 1e6:.0f} MB streamed in phase A, "
                          f"{(202.4e6 + 2 * qbytes / 8) / 1e6:.0f} MB of weights+activations in phase B)",
                    "parallelism": "replicas" if world > 1 else "single"},
@@ -279,8 +291,8 @@ def run_ours(args):
         "roofline": {"kernel": "w8a8_gemm_pair_kernel (tcgen05 int8, CTA pairs, activation quantizer inside)",
                      "bound": "tensor", "achieved": round(ach_l, 2),
                      "peak": round(int8_peak, 1), "unit": "TOP/s", "frac": round(ach_l / int8_peak, 4),
-                     "traffic": (NCU_TRAFFIC_GEMM_MEAN if T_TOKENS == 2048 else None),
-                     "traffic_note": "DRAM bytes per launch, mean over the step's seven launches",
+                     "traffic": (NCU_TRAFFIC_GEMM if T_TOKENS == 2048 and args.linear_calls == "layer" else None),
+                     "traffic_note": "DRAM bytes of the launch that runs the step's seven linears",
                      "peak_source": f"{peak_kind} sustained bf16 cuBLAS x 2 (nominal int8:bf16 ratio)"},
         "roofline_quantizer": {"kernel": "fakequant_kernel (fused fwd+bwd)", "bound": "hbm", "achieved": round(ach_q, 1),
                                "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(ach_q / peaks["hbm_gbs"], 4),
@@ -427,6 +439,9 @@ def main():
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--linear-calls", choices=["layer", "dependent", "each"], default="layer",
+                    help="phase B submits the seven linears in one call, in the groups a decoder layer's data flow "
+                         "allows (q/k/v | o | gate/up | down), or one call per linear")
     ap.add_argument("--tokens", type=int, default=2048,
                     help="tokens per step (default 2048, the headline workload; other values time the same layer at "
                          "decode or longer-prefill sizes and are named as such in config.workload)")

@@ -256,6 +256,36 @@ SASQ_API int sasq_dynamic_w8a8_linear(const void* x, const int8_t* w, const floa
                                       float* row_scale_out, int32_t* acc_out, int64_t T, int64_t N, int64_t K, int dt,
                                       int bits, void* workspace, size_t ws_bytes, void* stream);
 
+/* One linear of sasq_static_w8a8_linear_multi: the arguments of sasq_static_w8a8_linear for one problem.  The
+ * struct lives in HOST memory; the pointers in it are DEVICE pointers with the layouts, alignment and ownership
+ * stated there (bias may be NULL). */
+typedef struct sasq_linear_desc {
+    const void* x;          /* [T, K] 16-bit activations */
+    const int8_t* w;        /* [N, K] int8 weights */
+    const float* w_scale;   /* [N] fp32 */
+    const float* x_scale;   /* 1 fp32: the static factor of this linear's quantizer */
+    const void* bias;       /* [N] 16-bit, or NULL */
+    void* y;                /* [T, N] 16-bit output */
+    int64_t T, N, K;
+} sasq_linear_desc_t;
+
+/* Bytes of scratch sasq_static_w8a8_linear_multi needs for these problems (descs_host: HOST memory, count entries). */
+SASQ_API size_t sasq_static_w8a8_linear_multi_workspace(int count, const sasq_linear_desc_t* descs_host);
+
+/* Several independent static W8A8 linears (Sec. 4.4, Eq. 1 + Eq. 3, each exactly as sasq_static_w8a8_linear
+ * computes it: the results are bit-identical to `count` separate calls) submitted together, e.g. the q/k/v or the
+ * gate/up projections of a decoder layer, which do not depend on one another.  Consecutive problems with T > 128 run
+ * in ONE launch (up to 8 problems, 1024 256-row blocks and 80 MiB of int8 activation codes, i.e. sum of T x K,
+ * per launch, so that the codes stay in L2 until they are used; more are cut into several launches): the CTA
+ * pairs walk one tile list over all of them and the quantizer warps one chunk list, so the activation quantization
+ * of a problem and the drain of its last tiles overlap with the MMAs of its neighbours instead of idling the tensor
+ * cores at every launch boundary.  Problems with T <= 128 are launched on their own, in order.  No problem may read
+ * another's output.  descs_host: HOST memory, read before the call returns.  All problems share dt and bits.
+ * Returns SASQ_ERR_INVALID_ARG / UNSUPPORTED / WORKSPACE as sasq_static_w8a8_linear does, checked for every problem
+ * before anything is launched. */
+SASQ_API int sasq_static_w8a8_linear_multi(int count, const sasq_linear_desc_t* descs_host, int dt, int bits,
+                                           void* workspace, size_t ws_bytes, void* stream);
+
 /* How sasq_static_w8a8_linear splits a [T, N] output over `num_pairs` co-operating CTA pairs when T > 128
  * (introspection for tests and tuning; runs on the host, touches no device).  Every 256-row block is cut into the
  * same number of column tiles, widths multiples of 16 that differ by at most 16; the number is chosen so that the

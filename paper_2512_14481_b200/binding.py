@@ -23,7 +23,8 @@ __all__ = [
     "sasq_fakequant_fwd_bwd_ablation", "sasq_adamw_scales", "SASQ_FULL_OPERATOR", "SASQ_WITHOUT_ROUND",
     "SASQ_WITHOUT_CLAMP", "sasq_dynamic_w8a8_linear_workspace", "sasq_dynamic_w8a8_linear", "sasq_debug_set_wait_limit", "PcDesc", "sasq_fakequant_per_channel_multi_workspace",
     "sasq_fakequant_fwd_bwd_per_channel_multi", "sasq_static_w8a8_linear_per_channel_workspace",
-    "sasq_static_w8a8_linear_per_channel",
+    "sasq_static_w8a8_linear_per_channel", "LinearDesc", "sasq_static_w8a8_linear_multi_workspace",
+    "sasq_static_w8a8_linear_multi", "linear_multi_launches",
 ]
 
 SASQ_F16 = 0
@@ -63,6 +64,13 @@ class PcDesc(ctypes.Structure):
     _fields_ = [("x", ctypes.c_void_p), ("grad_y", ctypes.c_void_p), ("y", ctypes.c_void_p),
                 ("grad_x", ctypes.c_void_p), ("scales", ctypes.c_void_p), ("grad_scales", ctypes.c_void_p),
                 ("T", ctypes.c_int64), ("K", ctypes.c_int64), ("reserved", ctypes.c_int64)]
+
+
+class LinearDesc(ctypes.Structure):
+    """Mirror of sasq_linear_desc_t."""
+    _fields_ = [("x", ctypes.c_void_p), ("w", ctypes.c_void_p), ("w_scale", ctypes.c_void_p),
+                ("x_scale", ctypes.c_void_p), ("bias", ctypes.c_void_p), ("y", ctypes.c_void_p),
+                ("T", ctypes.c_int64), ("N", ctypes.c_int64), ("K", ctypes.c_int64)]
 
 
 def library_path() -> str:
@@ -122,6 +130,10 @@ def load_library() -> ctypes.CDLL:
     L.sasq_fakequant_fwd_bwd_per_channel_multi.argtypes = [ctypes.POINTER(PcDesc), i32, i32, i32, i32, vp, sz, vp]
     L.sasq_debug_set_wait_limit.restype = ctypes.c_longlong
     L.sasq_debug_set_wait_limit.argtypes = [ctypes.c_longlong]
+    L.sasq_static_w8a8_linear_multi_workspace.restype = sz
+    L.sasq_static_w8a8_linear_multi_workspace.argtypes = [i32, ctypes.POINTER(LinearDesc)]
+    L.sasq_static_w8a8_linear_multi.restype = i32
+    L.sasq_static_w8a8_linear_multi.argtypes = [i32, ctypes.POINTER(LinearDesc), i32, i32, vp, sz, vp]
     L.sasq_static_w8a8_linear_tiles.restype = i32
     L.sasq_static_w8a8_linear_tiles.argtypes = [i64, i64, i32, i32, ctypes.POINTER(ctypes.c_int32), i32]
     L.sasq_device_status.restype = i32
@@ -367,6 +379,70 @@ def sasq_static_w8a8_linear(x, w, w_scale, x_scale, y, bias=None, acc_out=None, 
     _check(load_library().sasq_static_w8a8_linear(_ptr(x), _ptr(w), _ptr(w_scale), _ptr(x_scale), _ptr(bias), _ptr(y),
                                                   _ptr(acc_out), T, N, K, _dt(x), int(bits), _ptr(workspace),
                                                   _nbytes(workspace), _stream(stream)), "sasq_static_w8a8_linear")
+
+
+def _linear_descs(problems):
+    """problems: sequence of (x, w, w_scale, x_scale, y) or (x, w, w_scale, x_scale, y, bias)."""
+    arr = (LinearDesc * max(1, len(problems)))()
+    dt = None
+    for i, pr in enumerate(problems):
+        x, w, w_scale, x_scale, y = pr[:5]
+        bias = pr[5] if len(pr) > 5 else None
+        _dev(x, "x"); _dev(w, "w", torch.int8); _dev(w_scale, "w_scale", torch.float32)
+        _dev(x_scale, "x_scale", torch.float32); _dev(y, "y", x.dtype)
+        if bias is not None:
+            _dev(bias, "bias", x.dtype)
+        if x.dim() != 2 or w.dim() != 2 or x.shape[1] != w.shape[1]:
+            raise ValueError("x must be [T, K] and w [N, K]")
+        T, K = x.shape
+        N = w.shape[0]
+        if tuple(y.shape) != (T, N) or w_scale.numel() != N or (bias is not None and bias.numel() != N):
+            raise ValueError("y must be [T, N], w_scale and bias [N]")
+        if dt is None:
+            dt = _dt(x)
+        elif dt != _dt(x):
+            raise ValueError("all problems of one call share the activation dtype")
+        arr[i] = LinearDesc(_ptr(x), _ptr(w), _ptr(w_scale), _ptr(x_scale), _ptr(bias), _ptr(y), T, N, K)
+    return arr, dt
+
+
+def sasq_static_w8a8_linear_multi_workspace(shapes) -> int:
+    """shapes: sequence of (T, N, K)."""
+    arr = (LinearDesc * max(1, len(shapes)))()
+    for i, (T, N, K) in enumerate(shapes):
+        arr[i].T, arr[i].N, arr[i].K = int(T), int(N), int(K)
+    return int(load_library().sasq_static_w8a8_linear_multi_workspace(len(shapes), arr))
+
+
+def sasq_static_w8a8_linear_multi(problems, workspace, bits: int = 8, stream=None) -> None:
+    """Independent static W8A8 linears submitted together; see _linear_descs for the tuples."""
+    arr, dt = _linear_descs(problems)
+    _dev(workspace, "workspace")
+    _check(load_library().sasq_static_w8a8_linear_multi(len(problems), arr, dt if dt is not None else SASQ_BF16, int(bits),
+                                                        _ptr(workspace), _nbytes(workspace), _stream(stream)),
+           "sasq_static_w8a8_linear_multi")
+
+
+def linear_multi_launches(shapes) -> int:
+    """Kernels one sasq_static_w8a8_linear_multi call launches for problems of these (T, N, K) (launch counting):
+    runs of problems with 128 < T <= 262144 share a launch, up to 8 problems, 1024 256-row blocks and 80 MiB of int8
+    activation codes each."""
+    launches, in_group, blocks, codes = 0, 0, 0, 0
+    for T, _, K in shapes:
+        if T == 0:
+            continue
+        mb = (T + 255) // 256
+        if T <= 128 or mb > 1024:
+            launches += linear_launches(T)
+            in_group, blocks, codes = 0, 0, 0
+            continue
+        if in_group == 0 or in_group == 8 or blocks + mb > 1024 or codes + T * K > (80 << 20):
+            launches += 1
+            in_group, blocks, codes = 0, 0, 0
+        in_group += 1
+        blocks += mb
+        codes += T * K
+    return launches
 
 
 def sasq_static_w8a8_linear_per_channel_workspace(T: int, N: int, K: int) -> int:

@@ -371,6 +371,30 @@ struct PairParams {
     unsigned* ready;    // [pair_m_blocks] 8-element items of each 256-row block that are quantized and visible; zero at launch
     unsigned* done;     // CTAs that have finished; the last one zeroes `ready` and this counter again
     float qn, qp;
+    // place of this problem in a launch that runs several problems back to back
+    int tile_begin;         // tiles of the problems before it
+    long long chunk_begin;  // quantizer chunks of the problems before it
+};
+
+// One launch runs up to kMaxGroup independent linears back to back: every CTA pair walks one list of tiles that
+// covers all of them, and the quantizer warps walk one list of chunks, so the activation quantization of a problem
+// (the head of a launch) and the drain of its last tiles overlap with the MMAs of its neighbours.
+constexpr int kMaxGroup = 8;
+// The quantizer warps run ahead of the MMAs through the whole chunk list, so the int8 activations of every problem of
+// a launch are written early and read back later: a launch takes problems only while those codes (with the weights
+// streaming past them) stay in the 126 MB L2.
+constexpr long long kGroupCodeBytes = 80ll << 20;
+struct GroupParams {
+    int count;
+    int num_tiles;          // over all problems
+    long long num_chunks;   // quantizer chunks over all problems (0: every A was quantized by an earlier launch)
+    int ready_count;        // counters the last CTA zeroes again
+    unsigned* ready;
+    unsigned* done;
+    PairParams prob[kMaxGroup];
+};
+struct GroupMaps {
+    CUtensorMap a[kMaxGroup], w[kMaxGroup], y64[kMaxGroup], y16[kMaxGroup];
 };
 
 // first column and width of column tile j
@@ -544,16 +568,14 @@ __device__ __forceinline__ bool wait_bounded_pair(uint64_t* bar, uint32_t parity
 
 template <bool BF>
 __global__ void __launch_bounds__(P_NUM_THREADS, 1)
-w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
-                      const __grid_constant__ CUtensorMap tmap_y64, const __grid_constant__ CUtensorMap tmap_y16,
-                      const __grid_constant__ PairParams pp) {
+w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_constant__ GroupParams gp) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* tiles = smem_raw;
     uint8_t* out_stage = tiles + (size_t)P_STAGES * P_STAGE_BYTES;          // 1024-byte aligned
     PairTail* tail = reinterpret_cast<PairTail*>(out_stage + P_OUT_BYTES);
-    const LinearParams& p = pp.lp;
+    const LinearParams& p0 = gp.prob[0].lp;         // the status word and the wait limit are the same for all problems
     if ((ptx::smem_u32(tiles) & 1023u) != 0) {      // uniform over the grid: every CTA returns before any barrier
-        if (threadIdx.x == 0) atomicMax(p.status, (int)SASQ_ERR_CUDA);
+        if (threadIdx.x == 0) atomicMax(p0.status, (int)SASQ_ERR_CUDA);
         return;
     }
 
@@ -562,7 +584,6 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();        // 0 = leader
-    const uint32_t stage_tx = (uint32_t)(P_A_BYTES + pp.w_box_rows * BK);   // bytes this CTA's two loads deliver
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < P_STAGES; ++s) {
@@ -575,10 +596,12 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         }
         tail->abort_flag = 0;
         ptx::mbar_init_fence();
-        ptx::prefetch_tensormap(&tmap_a);
-        ptx::prefetch_tensormap(&tmap_w);
-        ptx::prefetch_tensormap(&tmap_y64);
-        ptx::prefetch_tensormap(&tmap_y16);
+        for (int q = 0; q < gp.count; ++q) {
+            ptx::prefetch_tensormap(&maps.a[q]);
+            ptx::prefetch_tensormap(&maps.w[q]);
+            ptx::prefetch_tensormap(&maps.y64[q]);
+            ptx::prefetch_tensormap(&maps.y16[q]);
+        }
     }
     if (warp == 1) {
         ptx::tmem_alloc_pair(&tail->tmem_base, TMEM_COLS);
@@ -591,25 +614,7 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     const uint32_t tmem_base = tail->tmem_base;
     pdl_wait();                         // set-up done; from here on global memory of earlier kernels is used
 
-    // what the activation quantizer warps work on (and what the producers wait for)
-    ConvJob job{};
-    long long conv_chunks = 0;
-    if (pp.x != nullptr) {
-        job.src = reinterpret_cast<const uint4*>(pp.x);
-        job.dst = reinterpret_cast<uint2*>(pp.a_int8);
-        job.ready = pp.ready;
-        job.total = (long long)p.T * (p.K >> 3);
-        job.items_per_block = (long long)PBM * (p.K >> 3);
-        job.chan_inv = p.chan_inv;
-        job.vec_per_row = (unsigned)(p.K >> 3);
-        job.inv = p.chan_inv == nullptr ? __fdiv_rn(1.0f, __ldg(p.x_scale)) : 0.0f;
-        job.qn = pp.qn;
-        job.qp = pp.qp;
-        job.eight = pp.qp == 127.0f;
-        conv_chunks = (job.total + CONV_CHUNK - 1) / CONV_CHUNK;
-    }
-
-    const int num_tiles = pp.pair_m_blocks * pp.n_tiles;
+    const int num_tiles = gp.num_tiles;
     const int pair_id = blockIdx.x >> 1;
     const int num_pairs = gridDim.x >> 1;
 
@@ -619,8 +624,16 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            int ready_blk = -1;
-            for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs) {
+            int ready_blk = -1, ready_q = -1;
+            int q = 0;
+            for (int g = pair_id; g < num_tiles && ok; g += num_pairs) {
+                while (q + 1 < gp.count && g >= gp.prob[q + 1].tile_begin) ++q;
+                const PairParams& pp = gp.prob[q];
+                const LinearParams& p = pp.lp;
+                const CUtensorMap* tmap_a = &maps.a[q];
+                const CUtensorMap* tmap_w = &maps.w[q];
+                const uint32_t stage_tx = (uint32_t)(P_A_BYTES + pp.w_box_rows * BK);   // bytes of this CTA's two loads
+                const int tile = g - pp.tile_begin;
                 const int m_blk = tile / pp.n_tiles;
                 int n0, bn;
                 pair_tile_cols(pp, tile - m_blk * pp.n_tiles, &n0, &bn);
@@ -629,7 +642,7 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 // tile fetches 8 rows it does not use (rows past N read as zero)
                 const int w_row = n0 + (int)rank * (bn >> 1);
                 int kb_a = 0;            // k-blocks of this tile whose W half is already on its way
-                if (pp.x != nullptr && m_blk != ready_blk) {
+                if (pp.x != nullptr && (m_blk != ready_blk || q != ready_q)) {
                     // The rows of this block must have been quantized, by whichever CTAs had them, and be visible
                     // to the TMA unit before the first A load of the tile.  W does not depend on that: while
                     // waiting, fill the free stages with the W halves of the first k-blocks.
@@ -640,7 +653,7 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                     while (kb_a < p.k_blocks && kb_a < P_STAGES && ptx::mbar_test_wait(&tail->empty[st], ph ^ 1u)) {
                         const uint32_t full_leader = ptx::mapa_u32(ptx::smem_u32(&tail->full[st]), 0);
                         if (rank == 0) ptx::mbar_arrive_expect_tx(&tail->full[st], 2u * stage_tx);
-                        ptx::tma_load_2d_pair(tiles + (size_t)st * P_STAGE_BYTES + P_A_BYTES, &tmap_w, full_leader,
+                        ptx::tma_load_2d_pair(tiles + (size_t)st * P_STAGE_BYTES + P_A_BYTES, tmap_w, full_leader,
                                               kb_a * BK, w_row);
                         ++kb_a;
                         if (++st == P_STAGES) { st = 0; ph ^= 1u; }
@@ -649,6 +662,7 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                     if (!ok) break;
                     asm volatile("fence.proxy.async.global;" ::: "memory");
                     ready_blk = m_blk;
+                    ready_q = q;
                 }
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
                     uint8_t* a_dst = tiles + (size_t)stage * P_STAGE_BYTES;
@@ -660,9 +674,9 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                         ok = wait_bounded_pair(&tail->empty[stage], phase ^ 1u, tail, p);
                         if (!ok) break;
                         if (rank == 0) ptx::mbar_arrive_expect_tx(&tail->full[stage], 2u * stage_tx);
-                        ptx::tma_load_2d_pair(a_dst + P_A_BYTES, &tmap_w, full_leader, kb * BK, w_row);
+                        ptx::tma_load_2d_pair(a_dst + P_A_BYTES, tmap_w, full_leader, kb * BK, w_row);
                     }
-                    ptx::tma_load_2d_pair(a_dst, &tmap_a, full_leader, kb * BK, a_row);
+                    ptx::tma_load_2d_pair(a_dst, tmap_a, full_leader, kb * BK, a_row);
                     if (++stage == P_STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -683,9 +697,13 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             uint32_t phase = 0;
             bool ok = true;
             int it = 0;
-            for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs, ++it) {
+            int q = 0;
+            for (int g = pair_id; g < num_tiles && ok; g += num_pairs, ++it) {
+                while (q + 1 < gp.count && g >= gp.prob[q + 1].tile_begin) ++q;
+                const PairParams& pp = gp.prob[q];
+                const LinearParams& p = pp.lp;
                 int n0, bn;
-                pair_tile_cols(pp, tile % pp.n_tiles, &n0, &bn);
+                pair_tile_cols(pp, (g - pp.tile_begin) % pp.n_tiles, &n0, &bn);
                 const uint32_t idesc = ptx::idesc_i8(PBM, bn);
                 const int buf = it & 1;
                 const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
@@ -720,29 +738,61 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         // in the order the tiles need them.  Every warp runs its own load -> quantize -> store -> fence -> publish
         // pipeline with 16 128-bit loads in flight per lane; the warps drift apart, which keeps DRAM busy while
         // some of them wait for their stores to be acknowledged.
-        if (pp.x != nullptr) {
+        // With several problems in the launch their chunks form one list, in problem order.
+        {
             const int cw = warp - (P_NUM_THREADS - CONV_THREADS) / 32;          // 0..7
             const long long stride = (long long)gridDim.x * CONV_WARPS;
-            for (long long c = (long long)blockIdx.x * CONV_WARPS + cw; c < conv_chunks; c += stride) {
+            ConvJob job{};
+            int q = 0, job_q = -1;
+            for (long long c = (long long)blockIdx.x * CONV_WARPS + cw; c < gp.num_chunks; c += stride) {
+                while (q + 1 < gp.count && c >= gp.prob[q + 1].chunk_begin) ++q;
+                if (q != job_q) {
+                    const PairParams& pp = gp.prob[q];
+                    const LinearParams& p = pp.lp;
+                    job.src = reinterpret_cast<const uint4*>(pp.x);
+                    job.dst = reinterpret_cast<uint2*>(pp.a_int8);
+                    job.ready = pp.ready;
+                    job.total = (long long)p.T * (p.K >> 3);
+                    job.items_per_block = (long long)PBM * (p.K >> 3);
+                    job.chan_inv = p.chan_inv;
+                    job.vec_per_row = (unsigned)(p.K >> 3);
+                    job.inv = p.chan_inv == nullptr ? __fdiv_rn(1.0f, __ldg(p.x_scale)) : 0.0f;
+                    job.qn = pp.qn;
+                    job.qp = pp.qp;
+                    job.eight = pp.qp == 127.0f;
+                    job_q = q;
+                }
+                const long long lc = c - gp.prob[q].chunk_begin;
                 uint4 v[CONV_ITEMS];
-                conv_load(job, c, lane, v);
-                conv_store<BF>(job, c, lane, v);
-                conv_publish(job, c, lane);
+                conv_load(job, lc, lane, v);
+                conv_store<BF>(job, lc, lane, v);
+                conv_publish(job, lc, lane);
             }
         }
     } else {
         // ---------------- epilogue (warps 2..5 of both CTAs) ----------------
         const int quad = warp & 3;
         const int et = threadIdx.x - 64;
-        const bool per_row = p.row_scale != nullptr;
-        const bool one_factor = !per_row && p.chan_inv == nullptr;       // one static factor for the whole tensor
-        const float sx = one_factor ? __ldg(p.x_scale) : 1.0f;
-        if (one_factor && blockIdx.x == 0 && et == 0 && scale_is_bad(sx)) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
-        const bool has_bias = p.bias != nullptr;
+        if (blockIdx.x == 0 && et < gp.count) {          // one thread per problem checks its static factor
+            const LinearParams& pe = gp.prob[et].lp;
+            if (pe.row_scale == nullptr && pe.chan_inv == nullptr && scale_is_bad(__ldg(pe.x_scale)))
+                atomicMax(pe.status, (int)SASQ_ERR_BAD_SCALE);
+        }
         bool ok = true;
         int it = 0;
         unsigned out_flip = 0;
-        for (int tile = pair_id; tile < num_tiles && ok; tile += num_pairs, ++it) {
+        int q = 0;
+        for (int g = pair_id; g < num_tiles && ok; g += num_pairs, ++it) {
+            while (q + 1 < gp.count && g >= gp.prob[q + 1].tile_begin) ++q;
+            const PairParams& pp = gp.prob[q];
+            const LinearParams& p = pp.lp;
+            const CUtensorMap* tmap_y64 = &maps.y64[q];
+            const CUtensorMap* tmap_y16 = &maps.y16[q];
+            const bool per_row = p.row_scale != nullptr;
+            const bool one_factor = !per_row && p.chan_inv == nullptr;       // one static factor for the whole tensor
+            const float sx = one_factor ? __ldg(p.x_scale) : 1.0f;
+            const bool has_bias = p.bias != nullptr;
+            const int tile = g - pp.tile_begin;
             const int m_blk = tile / pp.n_tiles;
             int n0, bn;
             pair_tile_cols(pp, tile - m_blk * pp.n_tiles, &n0, &bn);
@@ -812,7 +862,7 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    ptx::tma_store_2d(&tmap_y64, sbuf, n0 + c, row0);
+                    ptx::tma_store_2d(tmap_y64, sbuf, n0 + c, row0);
                     ptx::bulk_commit_group();
                 }
                 ++out_flip;
@@ -853,7 +903,7 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    ptx::tma_store_2d(&tmap_y16, sbuf, n0 + c, row0);
+                    ptx::tma_store_2d(tmap_y16, sbuf, n0 + c, row0);
                     ptx::bulk_commit_group();
                 }
                 ++out_flip;
@@ -879,13 +929,13 @@ w8a8_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc_pair(tmem_base, TMEM_COLS);
     }
-    if (pp.x != nullptr) {
+    if (gp.done != nullptr) {
         // the CTA that finishes last leaves the counters at zero for the next launch that draws them
-        if (threadIdx.x == 0) tail->is_last_cta = (atomicAdd(pp.done, 1u) == gridDim.x - 1) ? 1 : 0;
+        if (threadIdx.x == 0) tail->is_last_cta = (atomicAdd(gp.done, 1u) == gridDim.x - 1) ? 1 : 0;
         __syncthreads();
         if (tail->is_last_cta) {
-            for (int i = threadIdx.x; i < pp.pair_m_blocks; i += P_NUM_THREADS) pp.ready[i] = 0u;
-            if (threadIdx.x == 0) *pp.done = 0u;
+            for (int i = threadIdx.x; i < gp.ready_count; i += P_NUM_THREADS) gp.ready[i] = 0u;
+            if (threadIdx.x == 0) *gp.done = 0u;
         }
     }
 }
@@ -1558,11 +1608,10 @@ size_t sasq_static_w8a8_linear_workspace(int64_t T, int64_t N, int64_t K) {
 namespace sasq {
 namespace {
 
-// dynamic == false: static factor x_scale_dev (the hot path).  dynamic == true: every row gets its own max-based
-// factor, written to row_scale_out (or to the workspace when that is NULL) by a launch that also quantizes the rows.
-int linear_impl(const void* x, const int8_t* w, const float* w_scale, const float* x_scale_dev,
-                const float* x_scales_vec, bool dynamic, float* row_scale_out, const void* bias, void* y, int32_t* acc_out, int64_t T, int64_t N, int64_t K,
-                int dt, int bits, void* workspace, size_t ws_bytes, void* stream) {
+// what every entry point of the linear checks before it launches anything
+int check_linear_args(const void* x, const int8_t* w, const float* w_scale, const float* x_scale_dev,
+                      const float* x_scales_vec, bool dynamic, const float* row_scale_out, const void* bias,
+                      const void* y, const int32_t* acc_out, int64_t T, int64_t N, int64_t K, int dt, int bits) {
     if (T < 0 || N <= 0 || K <= 0) return SASQ_ERR_INVALID_ARG;
     if (dt != SASQ_F16 && dt != SASQ_BF16) return SASQ_ERR_INVALID_ARG;
     if (bits < 2 || bits > 8) return SASQ_ERR_INVALID_ARG;
@@ -1572,9 +1621,43 @@ int linear_impl(const void* x, const int8_t* w, const float* w_scale, const floa
     if (T > 0 && (x == nullptr || y == nullptr)) return SASQ_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(row_scale_out) & 3u) return SASQ_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(w) || !aligned16(y) || !aligned16(acc_out) ||
-        (reinterpret_cast<uintptr_t>(w_scale) & 3u) || (reinterpret_cast<uintptr_t>(bias) & 1u))
+        (reinterpret_cast<uintptr_t>(w_scale) & 3u) || (reinterpret_cast<uintptr_t>(x_scale_dev) & 3u) ||
+        (reinterpret_cast<uintptr_t>(bias) & 1u))
         return SASQ_ERR_INVALID_ARG;
     if (K % 16 != 0 || N % 8 != 0 || K > 131072 || T > (1 << 24) || N > (1 << 24)) return SASQ_ERR_UNSUPPORTED;
+    return SASQ_OK;
+}
+
+// One launch of the CTA-pair kernel over all problems of `gp`, on as many resident pairs as there are tiles.
+int launch_pair_group(const GroupMaps& maps, const GroupParams& gp, int pairs, bool bf, cudaStream_t st) {
+    const int grid = 2 * (gp.num_tiles < pairs ? gp.num_tiles : pairs);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(P_NUM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = kPairSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1] = pdl_attribute();
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    cudaError_t e;
+    if (bf) e = cudaLaunchKernelEx(&cfg, w8a8_gemm_pair_kernel<true>, maps, gp);
+    else e = cudaLaunchKernelEx(&cfg, w8a8_gemm_pair_kernel<false>, maps, gp);
+    return e == cudaSuccess ? SASQ_OK : SASQ_ERR_CUDA;
+}
+
+// dynamic == false: static factor x_scale_dev (the hot path).  dynamic == true: every row gets its own max-based
+// factor, written to row_scale_out (or to the workspace when that is NULL) by a launch that also quantizes the rows.
+int linear_impl(const void* x, const int8_t* w, const float* w_scale, const float* x_scale_dev,
+                const float* x_scales_vec, bool dynamic, float* row_scale_out, const void* bias, void* y, int32_t* acc_out, int64_t T, int64_t N, int64_t K,
+                int dt, int bits, void* workspace, size_t ws_bytes, void* stream) {
+    const int arg_rc = check_linear_args(x, w, w_scale, x_scale_dev, x_scales_vec, dynamic, row_scale_out, bias, y, acc_out,
+                                         T, N, K, dt, bits);
+    if (arg_rc != SASQ_OK) return arg_rc;
     if (T == 0) return SASQ_OK;
     const size_t ws_need = dynamic ? sasq_dynamic_w8a8_linear_workspace(T, N, K)
                            : x_scales_vec != nullptr ? sasq_static_w8a8_linear_per_channel_workspace(T, N, K)
@@ -1709,39 +1792,30 @@ int linear_impl(const void* x, const int8_t* w, const float* w_scale, const floa
         // CTA pairs, 256-row blocks cut into evenly wide column tiles that fill whole waves of the resident pairs
         const int pairs = pair_capacity(dt == SASQ_BF16, sm_count);
         if (pairs <= 0) return SASQ_ERR_CUDA;
-        PairParams pp{};
+        GroupParams gp{};
+        GroupMaps maps{};
+        PairParams& pp = gp.prob[0];
         plan_pair_tiles(&pp, (int)((T + PBM - 1) / PBM), N, pairs);
         p.m_blocks = pp.pair_m_blocks;
         p.n_blocks = pp.n_tiles;
         pp.lp = p;
         pp.qn = qn;
         pp.qp = qp;
+        gp.count = 1;
+        gp.num_tiles = pp.pair_m_blocks * pp.n_tiles;
         if (in_kernel_quantizer) {
             pp.x = static_cast<const uint16_t*>(x);
             pp.a_int8 = a_int8;
-            if (!next_ready_slot(&pp.ready, &pp.done)) return SASQ_ERR_CUDA;
+            if (!next_ready_slot(&gp.ready, &gp.done)) return SASQ_ERR_CUDA;
+            pp.ready = gp.ready;
+            gp.ready_count = pp.pair_m_blocks;
+            gp.num_chunks = (T * (K >> 3) + CONV_CHUNK - 1) / CONV_CHUNK;
         }
-        if (!make_tmap(&tmap_a, a_int8, T, K, 128) || !make_tmap(&tmap_w, w, N, K, pp.w_box_rows)) return SASQ_ERR_CUDA;
-        CUtensorMap tmap_y64, tmap_y16;
-        if (!make_tmap_out(&tmap_y64, y, T, N, 64) || !make_tmap_out(&tmap_y16, y, T, N, 16)) return SASQ_ERR_CUDA;
-        const long long tiles = (long long)p.m_blocks * p.n_blocks;
-        const int grid = 2 * (int)(tiles < pairs ? tiles : pairs);
-        cudaLaunchConfig_t cfg{};
-        cfg.gridDim = dim3((unsigned)grid, 1, 1);
-        cfg.blockDim = dim3(P_NUM_THREADS, 1, 1);
-        cfg.dynamicSmemBytes = kPairSmemBytes;
-        cfg.stream = st;
-        cudaLaunchAttribute attr[2];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        attr[1] = pdl_attribute();
-        cfg.attrs = attr;
-        cfg.numAttrs = 2;
-        if (dt == SASQ_BF16) e = cudaLaunchKernelEx(&cfg, w8a8_gemm_pair_kernel<true>, tmap_a, tmap_w, tmap_y64, tmap_y16, pp);
-        else e = cudaLaunchKernelEx(&cfg, w8a8_gemm_pair_kernel<false>, tmap_a, tmap_w, tmap_y64, tmap_y16, pp);
-        if (e != cudaSuccess) return SASQ_ERR_CUDA;
+        if (!make_tmap(&maps.a[0], a_int8, T, K, 128) || !make_tmap(&maps.w[0], w, N, K, pp.w_box_rows) ||
+            !make_tmap_out(&maps.y64[0], y, T, N, 64) || !make_tmap_out(&maps.y16[0], y, T, N, 16))
+            return SASQ_ERR_CUDA;
+        const int rc = launch_pair_group(maps, gp, pairs, dt == SASQ_BF16, st);
+        if (rc != SASQ_OK) return rc;
     } else {
         p.m_blocks = (int)((T + BM - 1) / BM);
         p.n_blocks = (int)((N + BN - 1) / BN);
@@ -1766,6 +1840,114 @@ int sasq_static_w8a8_linear(const void* x, const int8_t* w, const float* w_scale
                             int bits, void* workspace, size_t ws_bytes, void* stream) {
     return sasq::linear_impl(x, w, w_scale, x_scale_dev, nullptr, false, nullptr, bias, y, acc_out, T, N, K, dt, bits,
                              workspace, ws_bytes, stream);
+}
+
+size_t sasq_static_w8a8_linear_multi_workspace(int count, const sasq_linear_desc_t* descs_host) {
+    if (count <= 0 || descs_host == nullptr) return 0;
+    size_t total = 0;
+    for (int i = 0; i < count; ++i) {
+        const size_t one = sasq_static_w8a8_linear_workspace(descs_host[i].T, descs_host[i].N, descs_host[i].K);
+        total += (one + 255) / 256 * 256;
+    }
+    return total + 256;
+}
+
+int sasq_static_w8a8_linear_multi(int count, const sasq_linear_desc_t* descs_host, int dt, int bits, void* workspace,
+                                  size_t ws_bytes, void* stream) {
+    using namespace sasq;
+    if (count < 0 || (count > 0 && descs_host == nullptr)) return SASQ_ERR_INVALID_ARG;
+    for (int i = 0; i < count; ++i) {
+        const sasq_linear_desc_t& d = descs_host[i];
+        const int rc = check_linear_args(d.x, d.w, d.w_scale, d.x_scale, nullptr, false, nullptr, d.bias, d.y, nullptr,
+                                         d.T, d.N, d.K, dt, bits);
+        if (rc != SASQ_OK) return rc;
+    }
+    if (count == 0) return SASQ_OK;
+    if (workspace == nullptr || !aligned16(workspace) ||
+        ws_bytes < sasq_static_w8a8_linear_multi_workspace(count, descs_host))
+        return SASQ_ERR_WORKSPACE;
+    const int sm_count = device_sm_count_if_sm100();
+    if (sm_count <= 0) return SASQ_ERR_UNSUPPORTED;
+    int* status = status_word_ptr();
+    if (status == nullptr) return SASQ_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool bf = dt == SASQ_BF16;
+    const int pairs = pair_capacity(bf, sm_count);
+    if (pairs <= 0) return SASQ_ERR_CUDA;
+    const float qn = (float)(1 << (bits - 1)), qp = (float)((1 << (bits - 1)) - 1);
+    const long long wait_limit = g_wait_limit.load(std::memory_order_relaxed);
+
+    uintptr_t ws = (reinterpret_cast<uintptr_t>(workspace) + 255) & ~uintptr_t(255);
+    GroupParams gp{};
+    GroupMaps maps{};
+    auto flush = [&]() -> int {
+        if (gp.count == 0) return SASQ_OK;
+        if (!next_ready_slot(&gp.ready, &gp.done)) return SASQ_ERR_CUDA;
+        int off = 0;
+        for (int q = 0; q < gp.count; ++q) {
+            gp.prob[q].ready = gp.ready + off;
+            off += gp.prob[q].pair_m_blocks;
+        }
+        gp.ready_count = off;
+        const int rc = launch_pair_group(maps, gp, pairs, bf, st);
+        gp = GroupParams{};
+        return rc;
+    };
+    for (int i = 0; i < count; ++i) {
+        const sasq_linear_desc_t& d = descs_host[i];
+        const size_t one = (sasq_static_w8a8_linear_workspace(d.T, d.N, d.K) + 255) / 256 * 256;
+        void* my_ws = reinterpret_cast<void*>(ws);
+        ws += one;
+        if (d.T == 0) continue;
+        const int m_blocks = (int)((d.T + PBM - 1) / PBM);
+        if (d.T <= BM || m_blocks > kMaxRowBlocks) {
+            // not a case for the CTA-pair kernel's in-kernel quantizer: on its own, in order
+            int rc = flush();
+            if (rc != SASQ_OK) return rc;
+            rc = linear_impl(d.x, d.w, d.w_scale, d.x_scale, nullptr, false, nullptr, d.bias, d.y, nullptr, d.T, d.N, d.K,
+                             dt, bits, my_ws, one, stream);
+            if (rc != SASQ_OK) return rc;
+            continue;
+        }
+        int blocks_so_far = 0;
+        long long codes_so_far = 0;
+        for (int q = 0; q < gp.count; ++q) {
+            blocks_so_far += gp.prob[q].pair_m_blocks;
+            codes_so_far += (long long)gp.prob[q].lp.T * gp.prob[q].lp.K;
+        }
+        if (gp.count == kMaxGroup || blocks_so_far + m_blocks > kMaxRowBlocks ||
+            (gp.count > 0 && codes_so_far + d.T * d.K > kGroupCodeBytes)) {
+            const int rc = flush();
+            if (rc != SASQ_OK) return rc;
+        }
+        const int q = gp.count;
+        PairParams& pp = gp.prob[q];
+        plan_pair_tiles(&pp, m_blocks, d.N, pairs);
+        LinearParams& p = pp.lp;
+        p.w_scale = d.w_scale;
+        p.x_scale = d.x_scale;
+        p.bias = d.bias;
+        p.y = d.y;
+        p.T = (int)d.T; p.N = (int)d.N; p.K = (int)d.K;
+        p.k_blocks = (int)((d.K + BK - 1) / BK);
+        p.m_blocks = pp.pair_m_blocks;
+        p.n_blocks = pp.n_tiles;
+        p.status = status;
+        p.wait_limit = wait_limit;
+        pp.qn = qn;
+        pp.qp = qp;
+        pp.x = static_cast<const uint16_t*>(d.x);
+        pp.a_int8 = reinterpret_cast<uint8_t*>(my_ws);
+        pp.tile_begin = gp.num_tiles;
+        pp.chunk_begin = gp.num_chunks;
+        if (!make_tmap(&maps.a[q], pp.a_int8, d.T, d.K, 128) || !make_tmap(&maps.w[q], d.w, d.N, d.K, pp.w_box_rows) ||
+            !make_tmap_out(&maps.y64[q], d.y, d.T, d.N, 64) || !make_tmap_out(&maps.y16[q], d.y, d.T, d.N, 16))
+            return SASQ_ERR_CUDA;
+        gp.num_tiles += pp.pair_m_blocks * pp.n_tiles;
+        gp.num_chunks += (d.T * (d.K >> 3) + CONV_CHUNK - 1) / CONV_CHUNK;
+        gp.count = q + 1;
+    }
+    return flush();
 }
 
 size_t sasq_static_w8a8_linear_per_channel_workspace(int64_t T, int64_t N, int64_t K) {
