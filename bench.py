@@ -184,7 +184,7 @@ class Layer:
         n = 0
         for call in self.calls:
             self.P.sasq_static_w8a8_linear_multi([self.linears[i] for i in call], self.l_ws, bits=BITS)
-            n += self.P.linear_multi_launches([self.shapes[i] for i in call])
+            n += self.P.sasq_static_w8a8_linear_multi_launches([self.shapes[i] for i in call])
         return n
 
 

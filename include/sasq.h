@@ -279,12 +279,19 @@ SASQ_API size_t sasq_static_w8a8_linear_multi_workspace(int count, const sasq_li
  * per launch, so that the codes stay in L2 until they are used; more are cut into several launches): the CTA
  * pairs walk one tile list over all of them and the quantizer warps one chunk list, so the activation quantization
  * of a problem and the drain of its last tiles overlap with the MMAs of its neighbours instead of idling the tensor
- * cores at every launch boundary.  Problems with T <= 128 are launched on their own, in order.  No problem may read
- * another's output.  descs_host: HOST memory, read before the call returns.  All problems share dt and bits.
+ * cores at every launch boundary.  A run that contains problems with T <= 128 shares a launch only if it has at
+ * least two problems whose output tiles fill every resident CTA pair (the weights then stream through one launch
+ * instead of one latency chain per linear); otherwise its problems are launched one by one, in order.  No problem
+ * may read another's output.  descs_host: HOST memory, read before the call returns.  All problems share dt and bits.
  * Returns SASQ_ERR_INVALID_ARG / UNSUPPORTED / WORKSPACE as sasq_static_w8a8_linear does, checked for every problem
  * before anything is launched. */
 SASQ_API int sasq_static_w8a8_linear_multi(int count, const sasq_linear_desc_t* descs_host, int dt, int bits,
                                            void* workspace, size_t ws_bytes, void* stream);
+
+/* How many kernels sasq_static_w8a8_linear_multi launches for these problems (only T, N, K of each descriptor are
+ * read) on a device with `num_pairs` resident CTA pairs (74 on a B200): introspection for launch counting and tests;
+ * runs on the host, touches no device.  Returns -1 for invalid arguments. */
+SASQ_API int sasq_static_w8a8_linear_multi_launches(int count, const sasq_linear_desc_t* descs_host, int num_pairs);
 
 /* How sasq_static_w8a8_linear splits a [T, N] output over `num_pairs` co-operating CTA pairs when T > 128
  * (introspection for tests and tuning; runs on the host, touches no device).  Every 256-row block is cut into the

@@ -24,7 +24,7 @@ __all__ = [
     "SASQ_WITHOUT_CLAMP", "sasq_dynamic_w8a8_linear_workspace", "sasq_dynamic_w8a8_linear", "sasq_debug_set_wait_limit", "PcDesc", "sasq_fakequant_per_channel_multi_workspace",
     "sasq_fakequant_fwd_bwd_per_channel_multi", "sasq_static_w8a8_linear_per_channel_workspace",
     "sasq_static_w8a8_linear_per_channel", "LinearDesc", "sasq_static_w8a8_linear_multi_workspace",
-    "sasq_static_w8a8_linear_multi", "linear_multi_launches",
+    "sasq_static_w8a8_linear_multi", "sasq_static_w8a8_linear_multi_launches",
 ]
 
 SASQ_F16 = 0
@@ -134,6 +134,8 @@ def load_library() -> ctypes.CDLL:
     L.sasq_static_w8a8_linear_multi_workspace.argtypes = [i32, ctypes.POINTER(LinearDesc)]
     L.sasq_static_w8a8_linear_multi.restype = i32
     L.sasq_static_w8a8_linear_multi.argtypes = [i32, ctypes.POINTER(LinearDesc), i32, i32, vp, sz, vp]
+    L.sasq_static_w8a8_linear_multi_launches.restype = i32
+    L.sasq_static_w8a8_linear_multi_launches.argtypes = [i32, ctypes.POINTER(LinearDesc), i32]
     L.sasq_static_w8a8_linear_tiles.restype = i32
     L.sasq_static_w8a8_linear_tiles.argtypes = [i64, i64, i32, i32, ctypes.POINTER(ctypes.c_int32), i32]
     L.sasq_device_status.restype = i32
@@ -423,26 +425,16 @@ def sasq_static_w8a8_linear_multi(problems, workspace, bits: int = 8, stream=Non
            "sasq_static_w8a8_linear_multi")
 
 
-def linear_multi_launches(shapes) -> int:
-    """Kernels one sasq_static_w8a8_linear_multi call launches for problems of these (T, N, K) (launch counting):
-    runs of problems with 128 < T <= 262144 share a launch, up to 8 problems, 1024 256-row blocks and 80 MiB of int8
-    activation codes each."""
-    launches, in_group, blocks, codes = 0, 0, 0, 0
-    for T, _, K in shapes:
-        if T == 0:
-            continue
-        mb = (T + 255) // 256
-        if T <= 128 or mb > 1024:
-            launches += linear_launches(T)
-            in_group, blocks, codes = 0, 0, 0
-            continue
-        if in_group == 0 or in_group == 8 or blocks + mb > 1024 or codes + T * K > (80 << 20):
-            launches += 1
-            in_group, blocks, codes = 0, 0, 0
-        in_group += 1
-        blocks += mb
-        codes += T * K
-    return launches
+def sasq_static_w8a8_linear_multi_launches(shapes, num_pairs: int = 74) -> int:
+    """Kernels one sasq_static_w8a8_linear_multi call launches for problems of these (T, N, K) on a device with
+    `num_pairs` resident CTA pairs (launch counting; asks the library, touches no device)."""
+    arr = (LinearDesc * max(1, len(shapes)))()
+    for i, (T, N, K) in enumerate(shapes):
+        arr[i].T, arr[i].N, arr[i].K = int(T), int(N), int(K)
+    n = int(load_library().sasq_static_w8a8_linear_multi_launches(len(shapes), arr, int(num_pairs)))
+    if n < 0:
+        raise ValueError("invalid shapes")
+    return n
 
 
 def sasq_static_w8a8_linear_per_channel_workspace(T: int, N: int, K: int) -> int:

@@ -1650,6 +1650,49 @@ int launch_pair_group(const GroupMaps& maps, const GroupParams& gp, int pairs, b
     return e == cudaSuccess ? SASQ_OK : SASQ_ERR_CUDA;
 }
 
+// Cuts a list of problems into runs that fit one launch of the CTA-pair kernel (up to kMaxGroup problems,
+// kMaxRowBlocks row blocks, kGroupCodeBytes of int8 codes) and tells `visit(first, last, grouped)` for each run
+// whether it goes to that kernel in one launch: yes if all its problems have T > 128, or if it has small-T problems
+// but at least two problems whose tiles fill every resident pair (the weights then stream through one launch
+// instead of one latency chain per linear); otherwise its problems are launched one by one, in order.
+template <typename Visit>
+int for_each_run(int count, const sasq_linear_desc_t* descs, int pairs, Visit visit) {
+    int first = 0;
+    while (first < count) {
+        int last = first, live = 0, blocks = 0, tiles = 0;
+        long long codes = 0;
+        bool small_t = false;
+        while (last < count) {
+            const sasq_linear_desc_t& d = descs[last];
+            if (d.T > 0) {
+                const long long m_blocks = (d.T + PBM - 1) / PBM;
+                if (m_blocks > kMaxRowBlocks) break;                 // on its own, below
+                if (live == kMaxGroup || blocks + m_blocks > kMaxRowBlocks ||
+                    (live > 0 && codes + d.T * d.K > kGroupCodeBytes))
+                    break;
+                PairParams plan{};
+                plan_pair_tiles(&plan, (int)m_blocks, d.N, pairs);
+                tiles += plan.pair_m_blocks * plan.n_tiles;
+                blocks += (int)m_blocks;
+                codes += d.T * d.K;
+                small_t = small_t || d.T <= BM;
+                ++live;
+            }
+            ++last;
+        }
+        int rc;
+        if (last == first) {                                          // a problem no launch can share
+            rc = visit(first, first + 1, false);
+            last = first + 1;
+        } else {
+            rc = visit(first, last, !small_t || (live >= 2 && tiles >= pairs));
+        }
+        if (rc != SASQ_OK) return rc;
+        first = last;
+    }
+    return SASQ_OK;
+}
+
 // dynamic == false: static factor x_scale_dev (the hot path).  dynamic == true: every row gets its own max-based
 // factor, written to row_scale_out (or to the workspace when that is NULL) by a launch that also quantizes the rows.
 int linear_impl(const void* x, const int8_t* w, const float* w_scale, const float* x_scale_dev,
@@ -1877,10 +1920,58 @@ int sasq_static_w8a8_linear_multi(int count, const sasq_linear_desc_t* descs_hos
     const float qn = (float)(1 << (bits - 1)), qp = (float)((1 << (bits - 1)) - 1);
     const long long wait_limit = g_wait_limit.load(std::memory_order_relaxed);
 
-    uintptr_t ws = (reinterpret_cast<uintptr_t>(workspace) + 255) & ~uintptr_t(255);
-    GroupParams gp{};
-    GroupMaps maps{};
-    auto flush = [&]() -> int {
+    // workspace slice of problem i: the slices follow one another, each a multiple of 256 bytes
+    const uintptr_t ws0 = (reinterpret_cast<uintptr_t>(workspace) + 255) & ~uintptr_t(255);
+    auto slice_bytes = [&](int i) -> size_t {
+        const sasq_linear_desc_t& d = descs_host[i];
+        return (sasq_static_w8a8_linear_workspace(d.T, d.N, d.K) + 255) / 256 * 256;
+    };
+    auto slice = [&](int i) -> void* {
+        uintptr_t at = ws0;
+        for (int j = 0; j < i; ++j) at += slice_bytes(j);
+        return reinterpret_cast<void*>(at);
+    };
+
+    auto run_alone = [&](int i) -> int {
+        const sasq_linear_desc_t& d = descs_host[i];
+        return linear_impl(d.x, d.w, d.w_scale, d.x_scale, nullptr, false, nullptr, d.bias, d.y, nullptr, d.T, d.N, d.K,
+                           dt, bits, slice(i), slice_bytes(i), stream);
+    };
+    // one launch of the CTA-pair kernel for problems [first, last)
+    auto run_group = [&](int first, int last) -> int {
+        GroupParams gp{};
+        GroupMaps maps{};
+        for (int i = first; i < last; ++i) {
+            if (descs_host[i].T == 0) continue;
+            const sasq_linear_desc_t& d = descs_host[i];
+            const int q = gp.count;
+            PairParams& pp = gp.prob[q];
+            plan_pair_tiles(&pp, (int)((d.T + PBM - 1) / PBM), d.N, pairs);
+            LinearParams& p = pp.lp;
+            p.w_scale = d.w_scale;
+            p.x_scale = d.x_scale;
+            p.bias = d.bias;
+            p.y = d.y;
+            p.T = (int)d.T; p.N = (int)d.N; p.K = (int)d.K;
+            p.k_blocks = (int)((d.K + BK - 1) / BK);
+            p.m_blocks = pp.pair_m_blocks;
+            p.n_blocks = pp.n_tiles;
+            p.status = status;
+            p.wait_limit = wait_limit;
+            pp.qn = qn;
+            pp.qp = qp;
+            pp.x = static_cast<const uint16_t*>(d.x);
+            pp.a_int8 = reinterpret_cast<uint8_t*>(slice(i));
+            pp.tile_begin = gp.num_tiles;
+            pp.chunk_begin = gp.num_chunks;
+            if (!make_tmap(&maps.a[q], pp.a_int8, d.T, d.K, 128) ||
+                !make_tmap(&maps.w[q], d.w, d.N, d.K, pp.w_box_rows) ||
+                !make_tmap_out(&maps.y64[q], d.y, d.T, d.N, 64) || !make_tmap_out(&maps.y16[q], d.y, d.T, d.N, 16))
+                return SASQ_ERR_CUDA;
+            gp.num_tiles += pp.pair_m_blocks * pp.n_tiles;
+            gp.num_chunks += (d.T * (d.K >> 3) + CONV_CHUNK - 1) / CONV_CHUNK;
+            gp.count = q + 1;
+        }
         if (gp.count == 0) return SASQ_OK;
         if (!next_ready_slot(&gp.ready, &gp.done)) return SASQ_ERR_CUDA;
         int off = 0;
@@ -1889,65 +1980,40 @@ int sasq_static_w8a8_linear_multi(int count, const sasq_linear_desc_t* descs_hos
             off += gp.prob[q].pair_m_blocks;
         }
         gp.ready_count = off;
-        const int rc = launch_pair_group(maps, gp, pairs, bf, st);
-        gp = GroupParams{};
-        return rc;
+        return launch_pair_group(maps, gp, pairs, bf, st);
     };
-    for (int i = 0; i < count; ++i) {
-        const sasq_linear_desc_t& d = descs_host[i];
-        const size_t one = (sasq_static_w8a8_linear_workspace(d.T, d.N, d.K) + 255) / 256 * 256;
-        void* my_ws = reinterpret_cast<void*>(ws);
-        ws += one;
-        if (d.T == 0) continue;
-        const int m_blocks = (int)((d.T + PBM - 1) / PBM);
-        if (d.T <= BM || m_blocks > kMaxRowBlocks) {
-            // not a case for the CTA-pair kernel's in-kernel quantizer: on its own, in order
-            int rc = flush();
-            if (rc != SASQ_OK) return rc;
-            rc = linear_impl(d.x, d.w, d.w_scale, d.x_scale, nullptr, false, nullptr, d.bias, d.y, nullptr, d.T, d.N, d.K,
-                             dt, bits, my_ws, one, stream);
-            if (rc != SASQ_OK) return rc;
-            continue;
+
+    return for_each_run(count, descs_host, pairs, [&](int first, int last, bool grouped) -> int {
+        if (grouped) return run_group(first, last);
+        int rc = SASQ_OK;
+        for (int i = first; i < last && rc == SASQ_OK; ++i) rc = run_alone(i);
+        return rc;
+    });
+}
+
+int sasq_static_w8a8_linear_multi_launches(int count, const sasq_linear_desc_t* descs_host, int num_pairs) {
+    using namespace sasq;
+    if (count < 0 || (count > 0 && descs_host == nullptr) || num_pairs <= 0) return -1;
+    for (int i = 0; i < count; ++i)
+        if (descs_host[i].T < 0 || descs_host[i].N <= 0 || descs_host[i].K <= 0) return -1;
+    int launches = 0;
+    for_each_run(count, descs_host, num_pairs, [&](int first, int last, bool grouped) -> int {
+        if (grouped) {
+            for (int i = first; i < last; ++i)
+                if (descs_host[i].T > 0) { ++launches; break; }
+            return SASQ_OK;
         }
-        int blocks_so_far = 0;
-        long long codes_so_far = 0;
-        for (int q = 0; q < gp.count; ++q) {
-            blocks_so_far += gp.prob[q].pair_m_blocks;
-            codes_so_far += (long long)gp.prob[q].lp.T * gp.prob[q].lp.K;
+        for (int i = first; i < last; ++i) {
+            const sasq_linear_desc_t& d = descs_host[i];
+            if (d.T == 0) continue;
+            // the activation quantizer runs inside the GEMM launch unless the row blocks (T > 128) or the
+            // 128-channel tiles (T <= 128) outnumber what its counters / the resident CTAs can hold
+            const bool inside = d.T > BM ? (d.T + PBM - 1) / PBM <= kMaxRowBlocks : (d.N + 127) / 128 <= 2 * num_pairs;
+            launches += inside ? 1 : 2;
         }
-        if (gp.count == kMaxGroup || blocks_so_far + m_blocks > kMaxRowBlocks ||
-            (gp.count > 0 && codes_so_far + d.T * d.K > kGroupCodeBytes)) {
-            const int rc = flush();
-            if (rc != SASQ_OK) return rc;
-        }
-        const int q = gp.count;
-        PairParams& pp = gp.prob[q];
-        plan_pair_tiles(&pp, m_blocks, d.N, pairs);
-        LinearParams& p = pp.lp;
-        p.w_scale = d.w_scale;
-        p.x_scale = d.x_scale;
-        p.bias = d.bias;
-        p.y = d.y;
-        p.T = (int)d.T; p.N = (int)d.N; p.K = (int)d.K;
-        p.k_blocks = (int)((d.K + BK - 1) / BK);
-        p.m_blocks = pp.pair_m_blocks;
-        p.n_blocks = pp.n_tiles;
-        p.status = status;
-        p.wait_limit = wait_limit;
-        pp.qn = qn;
-        pp.qp = qp;
-        pp.x = static_cast<const uint16_t*>(d.x);
-        pp.a_int8 = reinterpret_cast<uint8_t*>(my_ws);
-        pp.tile_begin = gp.num_tiles;
-        pp.chunk_begin = gp.num_chunks;
-        if (!make_tmap(&maps.a[q], pp.a_int8, d.T, d.K, 128) || !make_tmap(&maps.w[q], d.w, d.N, d.K, pp.w_box_rows) ||
-            !make_tmap_out(&maps.y64[q], d.y, d.T, d.N, 64) || !make_tmap_out(&maps.y16[q], d.y, d.T, d.N, 16))
-            return SASQ_ERR_CUDA;
-        gp.num_tiles += pp.pair_m_blocks * pp.n_tiles;
-        gp.num_chunks += (d.T * (d.K >> 3) + CONV_CHUNK - 1) / CONV_CHUNK;
-        gp.count = q + 1;
-    }
-    return flush();
+        return SASQ_OK;
+    });
+    return launches;
 }
 
 size_t sasq_static_w8a8_linear_per_channel_workspace(int64_t T, int64_t N, int64_t K) {

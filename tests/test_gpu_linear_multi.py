@@ -79,8 +79,9 @@ def test_single_problem_and_empty_call():
     assert P.sasq_device_status() == 0
 
 
-def test_small_t_and_empty_problems_between_grouped_ones():
-    """T <= 128 problems run on their own between two groups; a T = 0 problem is skipped; order is kept."""
+def test_small_t_and_empty_problems_between_larger_ones():
+    """A run with T <= 128 problems whose tiles do not fill the chip is launched problem by problem, in order; a
+    T = 0 problem is skipped."""
     tag = oracle.BF16
     problems = [make_problem(257, 256, 256, tag, 9300),
                 make_problem(64, 264, 144, tag, 9310),
@@ -88,14 +89,59 @@ def test_small_t_and_empty_problems_between_grouped_ones():
                 make_problem(1, 136, 528, tag, 9330, with_bias=True),
                 make_problem(384, 128, 1040, tag, 9340),
                 make_problem(200, 520, 96, tag, 9350)]
-    assert P.linear_multi_launches([(pr["T"], pr["N"], pr["K"]) for pr in problems]) == 4
+    assert P.sasq_static_w8a8_linear_multi_launches([(pr["T"], pr["N"], pr["K"]) for pr in problems]) == 5
     check_against_oracle(problems, tag)
+
+
+@pytest.mark.parametrize("tag", [oracle.F16, oracle.BF16])
+def test_small_t_problems_that_fill_the_chip_share_one_launch(tag):
+    """Decode-sized problems (T = 1, 16, 128) with enough output tiles for every CTA pair, and a T > 128 problem
+    among them, run in ONE launch of the CTA-pair kernel; every element against the oracle."""
+    problems = [make_problem(16, 11008, 256, tag, 9700),
+                make_problem(1, 4096, 144, tag, 9710, with_bias=True),
+                make_problem(128, 11008, 128, tag, 9720),
+                make_problem(300, 520, 96, tag, 9730),
+                make_problem(77, 4104, 64, tag, 9740)]
+    assert P.sasq_static_w8a8_linear_multi_launches([(pr["T"], pr["N"], pr["K"]) for pr in problems]) == 1
+    check_against_oracle(problems, tag)
+
+
+def test_llama7b_layer_at_decode_size_in_one_launch():
+    """The seven linears of a LLaMA-2-7B layer at T = 16: one launch, every output row against the oracle for three
+    of them, all seven bit-identical to separate calls (which take the small-T kernel)."""
+    tag, T = oracle.BF16, 16
+    probs, singles = [], []
+    for li, (name, K, N) in enumerate(W.LLAMA2_7B_LINEARS):
+        x = W.activations(T, K, torch.bfloat16, W.seed_of(3, 60 + li), device="cuda")
+        w = W.weights_fp32(N, K, W.seed_of(3, 70 + li), device="cuda")
+        w_int = torch.empty((N, K), dtype=torch.int8, device="cuda")
+        w_scale = torch.empty(N, dtype=torch.float32, device="cuda")
+        P.sasq_quantize_weight(w, w_int, w_scale, 8)
+        s = float(oracle.absmax_scale(oracle.bits_of(x.cpu())[0], tag, 8)) * W.learned_scale_factor(W.seed_of(3, li))
+        sc = torch.tensor([s], dtype=torch.float32, device="cuda")
+        y = torch.empty((T, N), dtype=torch.bfloat16, device="cuda")
+        probs.append((x, w_int, w_scale, sc, y))
+        y1 = torch.empty_like(y)
+        ws1 = torch.empty(P.sasq_static_w8a8_linear_workspace(T, N, K), dtype=torch.uint8, device="cuda")
+        P.sasq_static_w8a8_linear(x, w_int, w_scale, sc, y1, workspace=ws1)
+        singles.append((y1, s))
+    shapes = [(T, N, K) for _, K, N in W.LLAMA2_7B_LINEARS]
+    assert P.sasq_static_w8a8_linear_multi_launches(shapes) == 1
+    ws = torch.empty(P.sasq_static_w8a8_linear_multi_workspace(shapes), dtype=torch.uint8, device="cuda")
+    P.sasq_static_w8a8_linear_multi(probs, ws)
+    assert P.sasq_device_status() == 0
+    for li, ((x, w_int, w_scale, sc, y), (y1, s)) in enumerate(zip(probs, singles)):
+        assert torch.equal(y.view(torch.int16), y1.view(torch.int16)), li
+        if li in (0, 5, 6):
+            y_o, _, _ = oracle.w8a8_linear(oracle.bits_of(x.cpu())[0], tag, w_int.cpu().numpy(), w_scale.cpu().numpy(),
+                                           s, 8)
+            assert np.array_equal(host_bits(y), y_o), li
 
 
 def test_more_problems_than_one_launch_holds():
     tag = oracle.BF16
     problems = [make_problem(130 + 37 * i, 128 + 8 * i, 64 + 16 * i, tag, 9400 + 10 * i) for i in range(11)]
-    assert P.linear_multi_launches([(pr["T"], pr["N"], pr["K"]) for pr in problems]) == 2
+    assert P.sasq_static_w8a8_linear_multi_launches([(pr["T"], pr["N"], pr["K"]) for pr in problems]) == 2
     check_against_oracle(problems, tag)
 
 
@@ -129,7 +175,7 @@ def test_llama7b_layer_group_equals_separate_calls_and_oracle_rows():
         singles.append((y1, s))
     need = P.sasq_static_w8a8_linear_multi_workspace([(T, N, K) for _, K, N in W.LLAMA2_7B_LINEARS])
     ws = torch.empty(need, dtype=torch.uint8, device="cuda")
-    assert P.linear_multi_launches([(T, N, K) for _, K, N in W.LLAMA2_7B_LINEARS]) == 1
+    assert P.sasq_static_w8a8_linear_multi_launches([(T, N, K) for _, K, N in W.LLAMA2_7B_LINEARS]) == 1
     P.sasq_static_w8a8_linear_multi(probs, ws)
     assert P.sasq_device_status() == 0
     for li, ((x, w_int, w_scale, sc, y), (y1, s)) in enumerate(zip(probs, singles)):

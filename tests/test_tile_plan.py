@@ -50,3 +50,45 @@ def test_invalid_arguments():
     assert lib.sasq_static_w8a8_linear_tiles(0, 8, 4, 0, None, 0) == -1
     assert lib.sasq_static_w8a8_linear_tiles(256, 8, 4, 4, None, 0) == -1
     assert lib.sasq_static_w8a8_linear_tiles(256, 8, 0, 0, None, 0) == -1
+
+
+# ---------------------------------------------------------------------------
+# how sasq_static_w8a8_linear_multi cuts a list of problems into launches (host logic, no device)
+# ---------------------------------------------------------------------------
+LLAMA7B = [(4096, 4096)] * 4 + [(4096, 11008)] * 2 + [(11008, 4096)]          # (K, N) of the seven linears
+
+
+def launches(shapes, pairs=74):
+    return P.sasq_static_w8a8_linear_multi_launches(shapes, pairs)
+
+
+def test_multi_prefill_problems_share_launches_within_the_code_budget():
+    layer = lambda T: [(T, N, K) for K, N in LLAMA7B]
+    assert launches(layer(2048)) == 1            # 73 MB of int8 codes: one launch
+    assert launches(layer(129)) == 1
+    assert launches(layer(4096)) == 2            # 146 MB: cut where the running sum passes 80 MiB
+    assert launches(layer(16384)) == 7           # every problem's codes alone exceed the budget
+    assert launches([(300, 128, 64)] * 8) == 1 and launches([(300, 128, 64)] * 9) == 2     # 8 problems per launch
+    assert launches([(256 * 600, 128, 16)] * 2) == 2                                      # 1024 row blocks per launch
+    assert launches([]) == 0 and launches([(0, 128, 64)] * 3) == 0
+
+
+def test_multi_small_t_problems_share_a_launch_only_if_they_fill_the_chip():
+    layer = lambda T: [(T, N, K) for K, N in LLAMA7B]
+    for T in (1, 16, 128):
+        assert launches(layer(T)) == 1                       # 200+ tiles for 74 pairs
+        assert launches(layer(T)[:3]) == 3                   # q/k/v alone: about 60 tiles, one small-T launch each
+        assert launches(layer(T)[4:6]) == 1                  # gate/up: 106 tiles
+        assert launches(layer(T)[:1]) == 1
+    # a small-T problem whose 128-channel tiles outnumber the SMs needs a quantizer launch of its own
+    assert launches([(16, 19200, 80)]) == 2
+    # the same list on a (hypothetical) device with fewer resident pairs groups earlier
+    assert launches(layer(16)[:3], pairs=32) == 1
+
+
+def test_multi_launches_invalid_arguments():
+    import pytest
+    with pytest.raises(ValueError):
+        launches([(16, 0, 64)])
+    with pytest.raises(ValueError):
+        launches([(16, 128, 64)], pairs=0)
