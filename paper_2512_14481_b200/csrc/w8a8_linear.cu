@@ -778,6 +778,9 @@ w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
             if (pe.row_scale == nullptr && pe.chan_inv == nullptr && scale_is_bad(__ldg(pe.x_scale)))
                 atomicMax(pe.status, (int)SASQ_ERR_BAD_SCALE);
         }
+        // The outputs are not read again by this launch: their lines should leave L2 first, during the launch (whose
+        // DRAM interface is mostly idle), instead of staying behind dirty and being written back under the next kernel.
+        const uint64_t y_policy = ptx::l2_policy_evict_first();
         bool ok = true;
         int it = 0;
         unsigned out_flip = 0;
@@ -862,7 +865,7 @@ w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    ptx::tma_store_2d(tmap_y64, sbuf, n0 + c, row0);
+                    ptx::tma_store_2d_hint(tmap_y64, sbuf, n0 + c, row0, y_policy);
                     ptx::bulk_commit_group();
                 }
                 ++out_flip;
@@ -903,7 +906,7 @@ w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    ptx::tma_store_2d(tmap_y16, sbuf, n0 + c, row0);
+                    ptx::tma_store_2d_hint(tmap_y16, sbuf, n0 + c, row0, y_policy);
                     ptx::bulk_commit_group();
                 }
                 ++out_flip;
