@@ -24,7 +24,7 @@ __all__ = [
     "SASQ_WITHOUT_CLAMP", "sasq_dynamic_w8a8_linear_workspace", "sasq_dynamic_w8a8_linear", "sasq_debug_set_wait_limit", "PcDesc", "sasq_fakequant_per_channel_multi_workspace",
     "sasq_fakequant_fwd_bwd_per_channel_multi", "sasq_static_w8a8_linear_per_channel_workspace",
     "sasq_static_w8a8_linear_per_channel", "LinearDesc", "sasq_static_w8a8_linear_multi_workspace",
-    "sasq_static_w8a8_linear_multi", "sasq_static_w8a8_linear_multi_launches",
+    "sasq_static_w8a8_linear_multi", "sasq_static_w8a8_linear_multi_launches", "LinearProblems", "QuantTensors",
 ]
 
 SASQ_F16 = 0
@@ -237,31 +237,41 @@ def sasq_fakequant_multi_workspace(n_tensors: int) -> int:
     return int(load_library().sasq_fakequant_multi_workspace(int(n_tensors)))
 
 
+class QuantTensors:
+    """The descriptor table of a sasq_fakequant_fwd_bwd_multi call, marshalled once (see LinearProblems)."""
+
+    def __init__(self, tensors):
+        self.tensors = list(tensors)
+        n = len(self.tensors)
+        self.descs = (QDesc * max(n, 1))()
+        dt = None
+        for i, (x, gy, y, gx, idx) in enumerate(self.tensors):
+            _dev(x, "x")
+            for name, t in (("grad_y", gy), ("y", y), ("grad_x", gx)):
+                if t is not None:
+                    _dev(t, name, x.dtype)
+                    if t.numel() != x.numel():
+                        raise ValueError(f"{name} must have as many elements as x")
+            if dt is None:
+                dt = _dt(x)
+            elif dt != _dt(x):
+                raise TypeError("all tensors of one call must share a dtype")
+            self.descs[i] = QDesc(_ptr(x), _ptr(gy), _ptr(y), _ptr(gx), x.numel(), int(idx), 0)
+        self.dt = SASQ_BF16 if dt is None else dt
+        self.count = n
+
+
 def sasq_fakequant_fwd_bwd_multi(tensors, scales, grad_scales, workspace, bits: int = 8, accumulate: bool = False,
                                  stream=None) -> None:
-    """tensors: sequence of (x, grad_y | None, y | None, grad_x | None, scale_index)."""
-    n = len(tensors)
-    descs = (QDesc * max(n, 1))()
-    dt = None
-    for i, (x, gy, y, gx, idx) in enumerate(tensors):
-        _dev(x, "x")
-        for name, t in (("grad_y", gy), ("y", y), ("grad_x", gx)):
-            if t is not None:
-                _dev(t, name, x.dtype)
-                if t.numel() != x.numel():
-                    raise ValueError(f"{name} must have as many elements as x")
-        if dt is None:
-            dt = _dt(x)
-        elif dt != _dt(x):
-            raise TypeError("all tensors of one call must share a dtype")
-        descs[i] = QDesc(_ptr(x), _ptr(gy), _ptr(y), _ptr(gx), x.numel(), int(idx), 0)
+    """tensors: sequence of (x, grad_y | None, y | None, grad_x | None, scale_index), or a QuantTensors made from one."""
+    prepared = tensors if isinstance(tensors, QuantTensors) else QuantTensors(tensors)
     _dev(scales, "scales", torch.float32)
     if grad_scales is not None:
         _dev(grad_scales, "grad_scales", torch.float32)
     if workspace is not None:
         _dev(workspace, "workspace")
-    _check(load_library().sasq_fakequant_fwd_bwd_multi(descs, n, _ptr(scales), _ptr(grad_scales), scales.numel(),
-                                                       int(bool(accumulate)), SASQ_BF16 if dt is None else dt,
+    _check(load_library().sasq_fakequant_fwd_bwd_multi(prepared.descs, prepared.count, _ptr(scales), _ptr(grad_scales),
+                                                       scales.numel(), int(bool(accumulate)), prepared.dt,
                                                        int(bits), _ptr(workspace), _nbytes(workspace),
                                                        _stream(stream)), "sasq_fakequant_fwd_bwd_multi")
 
@@ -416,11 +426,24 @@ def sasq_static_w8a8_linear_multi_workspace(shapes) -> int:
     return int(load_library().sasq_static_w8a8_linear_multi_workspace(len(shapes), arr))
 
 
+class LinearProblems:
+    """The descriptor table of a sasq_static_w8a8_linear_multi call, marshalled once: a caller that submits the same
+    tensors again and again (a layer's weights and activation buffers) passes this instead of the tuples and skips
+    the per-call checks and conversions.  Holds references to the tensors so the pointers stay valid."""
+
+    def __init__(self, problems):
+        self.problems = list(problems)
+        self.descs, dt = _linear_descs(self.problems)
+        self.dt = SASQ_BF16 if dt is None else dt
+        self.count = len(self.problems)
+
+
 def sasq_static_w8a8_linear_multi(problems, workspace, bits: int = 8, stream=None) -> None:
-    """Independent static W8A8 linears submitted together; see _linear_descs for the tuples."""
-    arr, dt = _linear_descs(problems)
+    """Independent static W8A8 linears submitted together: a sequence of tuples (see _linear_descs) or a
+    LinearProblems made from one."""
+    prepared = problems if isinstance(problems, LinearProblems) else LinearProblems(problems)
     _dev(workspace, "workspace")
-    _check(load_library().sasq_static_w8a8_linear_multi(len(problems), arr, dt if dt is not None else SASQ_BF16, int(bits),
+    _check(load_library().sasq_static_w8a8_linear_multi(prepared.count, prepared.descs, prepared.dt, int(bits),
                                                         _ptr(workspace), _nbytes(workspace), _stream(stream)),
            "sasq_static_w8a8_linear_multi")
 

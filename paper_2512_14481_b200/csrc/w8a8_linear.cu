@@ -12,6 +12,7 @@
 //               so the quantization of later rows runs under the MMAs of earlier ones and costs no launch
 // Every wait on an mbarrier is bounded; a wait that gives up raises SASQ_ERR_TIMEOUT
 // in the sticky status word and all roles fall through to the teardown.
+#include <algorithm>
 #include <atomic>
 #include <mutex>
 
@@ -384,6 +385,13 @@ constexpr int kMaxGroup = 8;
 // a launch are written early and read back later: a launch takes problems only while those codes (with the weights
 // streaming past them) stay in the 126 MB L2.
 constexpr long long kGroupCodeBytes = 80ll << 20;
+// Which tiles a pair computes.  By default pair p takes tiles p, p + pairs, ... of the launch's tile list (column
+// tiles fastest, so the pairs of a wave share the rows of A and walk through W together).  When every problem has a
+// single 256-row block nothing is shared between tiles, and tiles of different problems cost very different amounts
+// (their K differs): the host then deals the tiles out by cost (longest first, always to the least loaded pair) and
+// passes each pair's list.
+constexpr int kMaxListTiles = 512;
+constexpr int kMaxListPairs = 96;
 struct GroupParams {
     int count;
     int num_tiles;          // over all problems
@@ -392,7 +400,31 @@ struct GroupParams {
     unsigned* ready;
     unsigned* done;
     PairParams prob[kMaxGroup];
+    int use_list;                                // 0: round-robin over the tile list; 1: the lists below
+    uint16_t list_begin[kMaxListPairs + 1];      // pair p computes tile_list[list_begin[p] .. list_begin[p + 1])
+    uint16_t tile_list[kMaxListTiles];
 };
+
+// the tiles of one pair, in the order it computes them
+struct TileWalk {
+    int at, end, step;
+    bool list;
+    __device__ __forceinline__ TileWalk(const GroupParams& gp, int pair_id, int num_pairs) {
+        list = gp.use_list != 0;
+        at = list ? (int)gp.list_begin[pair_id] : pair_id;
+        end = list ? (int)gp.list_begin[pair_id + 1] : gp.num_tiles;
+        step = list ? 1 : num_pairs;
+    }
+    __device__ __forceinline__ bool more() const { return at < end; }
+    __device__ __forceinline__ void next() { at += step; }
+    __device__ __forceinline__ int tile(const GroupParams& gp) const { return list ? (int)gp.tile_list[at] : at; }
+};
+// the problem tile g belongs to
+__device__ __forceinline__ int problem_of(const GroupParams& gp, int g) {
+    int q = 0;
+    while (q + 1 < gp.count && g >= gp.prob[q + 1].tile_begin) ++q;
+    return q;
+}
 struct GroupMaps {
     CUtensorMap a[kMaxGroup], w[kMaxGroup], y64[kMaxGroup], y16[kMaxGroup];
 };
@@ -614,7 +646,6 @@ w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
     const uint32_t tmem_base = tail->tmem_base;
     pdl_wait();                         // set-up done; from here on global memory of earlier kernels is used
 
-    const int num_tiles = gp.num_tiles;
     const int pair_id = blockIdx.x >> 1;
     const int num_pairs = gridDim.x >> 1;
 
@@ -625,9 +656,9 @@ w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
             uint32_t phase = 0;
             bool ok = true;
             int ready_blk = -1, ready_q = -1;
-            int q = 0;
-            for (int g = pair_id; g < num_tiles && ok; g += num_pairs) {
-                while (q + 1 < gp.count && g >= gp.prob[q + 1].tile_begin) ++q;
+            for (TileWalk walk(gp, pair_id, num_pairs); walk.more() && ok; walk.next()) {
+                const int g = walk.tile(gp);
+                const int q = problem_of(gp, g);
                 const PairParams& pp = gp.prob[q];
                 const LinearParams& p = pp.lp;
                 const CUtensorMap* tmap_a = &maps.a[q];
@@ -697,9 +728,9 @@ w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
             uint32_t phase = 0;
             bool ok = true;
             int it = 0;
-            int q = 0;
-            for (int g = pair_id; g < num_tiles && ok; g += num_pairs, ++it) {
-                while (q + 1 < gp.count && g >= gp.prob[q + 1].tile_begin) ++q;
+            for (TileWalk walk(gp, pair_id, num_pairs); walk.more() && ok; walk.next(), ++it) {
+                const int g = walk.tile(gp);
+                const int q = problem_of(gp, g);
                 const PairParams& pp = gp.prob[q];
                 const LinearParams& p = pp.lp;
                 int n0, bn;
@@ -784,9 +815,9 @@ w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
         bool ok = true;
         int it = 0;
         unsigned out_flip = 0;
-        int q = 0;
-        for (int g = pair_id; g < num_tiles && ok; g += num_pairs, ++it) {
-            while (q + 1 < gp.count && g >= gp.prob[q + 1].tile_begin) ++q;
+        for (TileWalk walk(gp, pair_id, num_pairs); walk.more() && ok; walk.next(), ++it) {
+            const int g = walk.tile(gp);
+            const int q = problem_of(gp, g);
             const PairParams& pp = gp.prob[q];
             const LinearParams& p = pp.lp;
             const CUtensorMap* tmap_y64 = &maps.y64[q];
@@ -1631,6 +1662,64 @@ int check_linear_args(const void* x, const int8_t* w, const float* w_scale, cons
     return SASQ_OK;
 }
 
+// When every problem of the launch has a single row block (nothing shared between tiles) and the lists fit the
+// parameter block, deal the tiles out by cost: longest first, each to the pair with the least work so far.  The cost
+// of a tile is its k-blocks (plus a few for the switch) times the MMA time of its width (one MMA of N columns keeps
+// the tensor pipe busy for about max(N, 208) / 2 cycles).  Leaves gp->use_list = 0 otherwise.
+void deal_tiles_by_cost(GroupParams* gp, int pairs) {
+    gp->use_list = 0;
+    const int np = gp->num_tiles < pairs ? gp->num_tiles : pairs;
+    if (gp->count < 2 || gp->num_tiles > kMaxListTiles || np > kMaxListPairs) return;
+    for (int q = 0; q < gp->count; ++q)
+        if (gp->prob[q].pair_m_blocks != 1) return;
+    struct Item { long long cost; int tile; };
+    Item items[kMaxListTiles];
+    int n = 0;
+    for (int q = 0; q < gp->count; ++q) {
+        const PairParams& pp = gp->prob[q];
+        for (int j = 0; j < pp.n_tiles; ++j) {
+            int n0, width;
+            pair_tile_cols(pp, j, &n0, &width);
+            items[n].cost = (long long)(pp.lp.k_blocks + 4) * (width > 208 ? width : 208);
+            items[n].tile = pp.tile_begin + j;
+            ++n;
+        }
+    }
+    std::stable_sort(items, items + n, [](const Item& a, const Item& b) { return a.cost > b.cost; });
+    // a binary min-heap of (load, pair): ties go to the lower pair index
+    struct Slot { long long load; int pair; };
+    Slot heap[kMaxListPairs];
+    for (int pr = 0; pr < np; ++pr) heap[pr] = Slot{0, pr};            // sorted, hence a heap
+    auto less = [](const Slot& a, const Slot& b) { return a.load < b.load || (a.load == b.load && a.pair < b.pair); };
+    int owner[kMaxListTiles];
+    int per_pair[kMaxListPairs] = {};
+    for (int i = 0; i < n; ++i) {
+        owner[i] = heap[0].pair;
+        ++per_pair[heap[0].pair];
+        heap[0].load += items[i].cost;
+        int at = 0;                                                    // sift the grown root down
+        for (;;) {
+            int least = at;
+            const int l = 2 * at + 1, r = l + 1;
+            if (l < np && less(heap[l], heap[least])) least = l;
+            if (r < np && less(heap[r], heap[least])) least = r;
+            if (least == at) break;
+            std::swap(heap[at], heap[least]);
+            at = least;
+        }
+    }
+    int at = 0;
+    for (int pr = 0; pr < np; ++pr) {
+        gp->list_begin[pr] = (uint16_t)at;
+        at += per_pair[pr];
+    }
+    gp->list_begin[np] = (uint16_t)at;
+    int fill[kMaxListPairs];
+    for (int pr = 0; pr < np; ++pr) fill[pr] = gp->list_begin[pr];
+    for (int i = 0; i < n; ++i) gp->tile_list[fill[owner[i]]++] = (uint16_t)items[i].tile;      // longest first
+    gp->use_list = 1;
+}
+
 // One launch of the CTA-pair kernel over all problems of `gp`, on as many resident pairs as there are tiles.
 int launch_pair_group(const GroupMaps& maps, const GroupParams& gp, int pairs, bool bf, cudaStream_t st) {
     const int grid = 2 * (gp.num_tiles < pairs ? gp.num_tiles : pairs);
@@ -1983,6 +2072,7 @@ int sasq_static_w8a8_linear_multi(int count, const sasq_linear_desc_t* descs_hos
             off += gp.prob[q].pair_m_blocks;
         }
         gp.ready_count = off;
+        deal_tiles_by_cost(&gp, pairs);
         return launch_pair_group(maps, gp, pairs, bf, st);
     };
 
