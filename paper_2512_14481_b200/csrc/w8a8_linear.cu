@@ -331,6 +331,15 @@ constexpr int P_STAGES = SASQ_PAIR_STAGES;
 constexpr int P_A_BYTES = 128 * BK;      // per CTA: 128 rows of A
 constexpr int P_B_BYTES_MAX = 128 * BK;  // per CTA: up to 128 rows of W
 constexpr int P_STAGE_BYTES = P_A_BYTES + P_B_BYTES_MAX;
+// A stage holds the CTA's half of the W tile first, then its rows of A.  The kernel exists in two layouts of the
+// same ring: 5 stages with all 128 rows of A, and, for launches whose problems all have T <= 32, 8 stages with 32
+// rows of A (only the leader CTA has rows below T and loads them; the MMA still reads 128 rows from each CTA's
+// shared memory, the rest being whatever lies behind, and the accumulator rows they produce are never stored).
+// Such launches stream the weights once and are bound by the weight bytes in flight: 8 x 15 KB instead of 5 x 15 KB
+// per CTA.
+constexpr int P_SMALL_ROWS = 32;
+constexpr int P_SMALL_STAGES = (P_STAGES * P_STAGE_BYTES) / (P_B_BYTES_MAX + P_SMALL_ROWS * BK);
+constexpr int P_MAX_STAGES = P_SMALL_STAGES > P_STAGES ? P_SMALL_STAGES : P_STAGES;
 
 constexpr int P_NUM_THREADS = 448;       // 14 warps: producer, MMA issuer, 4 epilogue, 8 activation quantizer
 constexpr int CONV_THREADS = 256;
@@ -344,8 +353,8 @@ constexpr int P_OUT_BUF_BYTES = 32 * 128;        // one epilogue warp's staging 
 constexpr int P_OUT_BYTES = 4 * 2 * P_OUT_BUF_BYTES;   // 4 warps, double buffered
 
 struct PairTail {
-    uint64_t full[P_STAGES];       // used in the leader: its producer arms it with the bytes of both CTAs' loads
-    uint64_t empty[P_STAGES];      // local: MMA of the pair has consumed the stage
+    uint64_t full[P_MAX_STAGES];   // used in the leader: its producer arms it with the bytes of both CTAs' loads
+    uint64_t empty[P_MAX_STAGES];  // local: MMA of the pair has consumed the stage
     uint64_t tmem_full[ACC_BUFS];  // local: accumulators of the tile are complete
     uint64_t tmem_empty[ACC_BUFS]; // used in the leader: 8 epilogue warps (4 per CTA) have drained the buffer
     float scale[256];
@@ -598,9 +607,14 @@ __device__ __forceinline__ bool wait_bounded_pair(uint64_t* bar, uint32_t parity
     return true;
 }
 
-template <bool BF>
+template <bool BF, bool SMALL>
 __global__ void __launch_bounds__(P_NUM_THREADS, 1)
 w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_constant__ GroupParams gp) {
+    constexpr int STAGES = SMALL ? P_SMALL_STAGES : P_STAGES;
+    constexpr int A_BYTES = SMALL ? P_SMALL_ROWS * BK : P_A_BYTES;
+    constexpr int STAGE_BYTES = P_B_BYTES_MAX + A_BYTES;
+    static_assert(STAGES * STAGE_BYTES <= P_STAGES * P_STAGE_BYTES, "both layouts use the same ring");
+    static_assert(STAGE_BYTES % 1024 == 0, "swizzled tiles start on 1024-byte boundaries");
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* tiles = smem_raw;
     uint8_t* out_stage = tiles + (size_t)P_STAGES * P_STAGE_BYTES;          // 1024-byte aligned
@@ -618,7 +632,7 @@ w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
     const uint32_t rank = ptx::cluster_ctarank();        // 0 = leader
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < P_STAGES; ++s) {
+        for (int s = 0; s < STAGES; ++s) {
             ptx::mbar_init(&tail->full[s], 1);
             ptx::mbar_init(&tail->empty[s], 1);
         }
@@ -663,7 +677,10 @@ w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
                 const LinearParams& p = pp.lp;
                 const CUtensorMap* tmap_a = &maps.a[q];
                 const CUtensorMap* tmap_w = &maps.w[q];
-                const uint32_t stage_tx = (uint32_t)(P_A_BYTES + pp.w_box_rows * BK);   // bytes of this CTA's two loads
+                // bytes both CTAs' loads deliver per stage: two halves of the W tile, and A from both (or, in the
+                // small layout, from the leader alone)
+                const uint32_t stage_tx = (uint32_t)(2 * pp.w_box_rows * BK + (SMALL ? A_BYTES : 2 * A_BYTES));
+                const bool load_a = !SMALL || rank == 0;
                 const int tile = g - pp.tile_begin;
                 const int m_blk = tile / pp.n_tiles;
                 int n0, bn;
@@ -681,13 +698,12 @@ w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
                     const unsigned need = (unsigned)((rows < PBM ? rows : PBM) * (p.K >> 3));
                     int st = stage;
                     uint32_t ph = phase;
-                    while (kb_a < p.k_blocks && kb_a < P_STAGES && ptx::mbar_test_wait(&tail->empty[st], ph ^ 1u)) {
+                    while (kb_a < p.k_blocks && kb_a < STAGES && ptx::mbar_test_wait(&tail->empty[st], ph ^ 1u)) {
                         const uint32_t full_leader = ptx::mapa_u32(ptx::smem_u32(&tail->full[st]), 0);
-                        if (rank == 0) ptx::mbar_arrive_expect_tx(&tail->full[st], 2u * stage_tx);
-                        ptx::tma_load_2d_pair(tiles + (size_t)st * P_STAGE_BYTES + P_A_BYTES, tmap_w, full_leader,
-                                              kb_a * BK, w_row);
+                        if (rank == 0) ptx::mbar_arrive_expect_tx(&tail->full[st], stage_tx);
+                        ptx::tma_load_2d_pair(tiles + (size_t)st * STAGE_BYTES, tmap_w, full_leader, kb_a * BK, w_row);
                         ++kb_a;
-                        if (++st == P_STAGES) { st = 0; ph ^= 1u; }
+                        if (++st == STAGES) { st = 0; ph ^= 1u; }
                     }
                     ok = wait_rows_ready(pp.ready + m_blk, need, tail, p);
                     if (!ok) break;
@@ -696,7 +712,7 @@ w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
                     ready_q = q;
                 }
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
-                    uint8_t* a_dst = tiles + (size_t)stage * P_STAGE_BYTES;
+                    uint8_t* w_dst = tiles + (size_t)stage * STAGE_BYTES;
                     // Only the leader arms the barrier (with the bytes of both CTAs); the partner's copies
                     // may complete first, which merely drives the transaction count negative for a while:
                     // the phase cannot complete before the leader's arrival.
@@ -704,11 +720,11 @@ w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
                     if (kb >= kb_a) {
                         ok = wait_bounded_pair(&tail->empty[stage], phase ^ 1u, tail, p);
                         if (!ok) break;
-                        if (rank == 0) ptx::mbar_arrive_expect_tx(&tail->full[stage], 2u * stage_tx);
-                        ptx::tma_load_2d_pair(a_dst + P_A_BYTES, tmap_w, full_leader, kb * BK, w_row);
+                        if (rank == 0) ptx::mbar_arrive_expect_tx(&tail->full[stage], stage_tx);
+                        ptx::tma_load_2d_pair(w_dst, tmap_w, full_leader, kb * BK, w_row);
                     }
-                    ptx::tma_load_2d_pair(a_dst, tmap_a, full_leader, kb * BK, a_row);
-                    if (++stage == P_STAGES) { stage = 0; phase ^= 1u; }
+                    if (load_a) ptx::tma_load_2d_pair(w_dst + P_B_BYTES_MAX, tmap_a, full_leader, kb * BK, a_row);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
             // after an abort, copies may still be in flight into this CTA's shared memory: their barrier lives in
@@ -722,8 +738,8 @@ w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
     } else if (warp == 1) {
         // ---------------- MMA issuer (leader CTA only) ----------------
         if (rank == 0 && ptx::elect_one()) {
-            const uint64_t a_desc0 = ptx::smem_desc_k_major_sw128(ptx::smem_u32(tiles));
-            const uint64_t b_desc0 = ptx::smem_desc_k_major_sw128(ptx::smem_u32(tiles) + P_A_BYTES);
+            const uint64_t a_desc0 = ptx::smem_desc_k_major_sw128(ptx::smem_u32(tiles) + P_B_BYTES_MAX);
+            const uint64_t b_desc0 = ptx::smem_desc_k_major_sw128(ptx::smem_u32(tiles));
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -748,8 +764,8 @@ w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
                     // 32 bytes of K per MMA inside the swizzled 128-byte row: +2 in the descriptor's address field
-                    const uint64_t a_desc = a_desc0 + (uint64_t)(stage * (P_STAGE_BYTES >> 4));
-                    const uint64_t b_desc = b_desc0 + (uint64_t)(stage * (P_STAGE_BYTES >> 4));
+                    const uint64_t a_desc = a_desc0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
+                    const uint64_t b_desc = b_desc0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
                     ptx::mma_i8_ss_pair(d_tmem, a_desc, b_desc, idesc, accumulate);
                     ptx::mma_i8_ss_pair_acc(d_tmem, a_desc + 2, b_desc + 2, idesc);
                     ptx::mma_i8_ss_pair_acc(d_tmem, a_desc + 4, b_desc + 4, idesc);
@@ -757,7 +773,7 @@ w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
                     accumulate = 1u;
                     ptx::mma_commit_pair(&tail->empty[stage], 0x3);          // stage reusable once these MMAs are done
                     if (kb == p.k_blocks - 1) ptx::mma_commit_pair(&tail->tmem_full[buf], 0x3);
-                    if (++stage == P_STAGES) { stage = 0; phase ^= 1u; }
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
         }
@@ -1490,9 +1506,12 @@ int pair_capacity(bool bf, int sm_count) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
     if (cache[dev][bf] != 0) return cache[dev][bf];
-    const void* fn = bf ? reinterpret_cast<const void*>(w8a8_gemm_pair_kernel<true>)
-                        : reinterpret_cast<const void*>(w8a8_gemm_pair_kernel<false>);
-    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemBytes) != cudaSuccess)
+    const void* fn = bf ? reinterpret_cast<const void*>(w8a8_gemm_pair_kernel<true, false>)
+                        : reinterpret_cast<const void*>(w8a8_gemm_pair_kernel<false, false>);
+    const void* fn_small = bf ? reinterpret_cast<const void*>(w8a8_gemm_pair_kernel<true, true>)
+                              : reinterpret_cast<const void*>(w8a8_gemm_pair_kernel<false, true>);
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(fn_small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemBytes) != cudaSuccess)
         return -1;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)sm_count, 1, 1);
@@ -1721,7 +1740,8 @@ void deal_tiles_by_cost(GroupParams* gp, int pairs) {
 }
 
 // One launch of the CTA-pair kernel over all problems of `gp`, on as many resident pairs as there are tiles.
-int launch_pair_group(const GroupMaps& maps, const GroupParams& gp, int pairs, bool bf, cudaStream_t st) {
+int launch_pair_group(const GroupMaps& maps, const GroupParams& gp, int pairs, bool bf, cudaStream_t st,
+                      bool small_layout = false) {
     const int grid = 2 * (gp.num_tiles < pairs ? gp.num_tiles : pairs);
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)grid, 1, 1);
@@ -1737,8 +1757,13 @@ int launch_pair_group(const GroupMaps& maps, const GroupParams& gp, int pairs, b
     cfg.attrs = attr;
     cfg.numAttrs = 2;
     cudaError_t e;
-    if (bf) e = cudaLaunchKernelEx(&cfg, w8a8_gemm_pair_kernel<true>, maps, gp);
-    else e = cudaLaunchKernelEx(&cfg, w8a8_gemm_pair_kernel<false>, maps, gp);
+    if (small_layout) {
+        if (bf) e = cudaLaunchKernelEx(&cfg, w8a8_gemm_pair_kernel<true, true>, maps, gp);
+        else e = cudaLaunchKernelEx(&cfg, w8a8_gemm_pair_kernel<false, true>, maps, gp);
+    } else {
+        if (bf) e = cudaLaunchKernelEx(&cfg, w8a8_gemm_pair_kernel<true, false>, maps, gp);
+        else e = cudaLaunchKernelEx(&cfg, w8a8_gemm_pair_kernel<false, false>, maps, gp);
+    }
     return e == cudaSuccess ? SASQ_OK : SASQ_ERR_CUDA;
 }
 
@@ -2033,6 +2058,8 @@ int sasq_static_w8a8_linear_multi(int count, const sasq_linear_desc_t* descs_hos
     auto run_group = [&](int first, int last) -> int {
         GroupParams gp{};
         GroupMaps maps{};
+        bool small_layout = true;               // every problem has at most 32 rows: the 8-stage layout
+        for (int i = first; i < last; ++i) small_layout = small_layout && descs_host[i].T <= P_SMALL_ROWS;
         for (int i = first; i < last; ++i) {
             if (descs_host[i].T == 0) continue;
             const sasq_linear_desc_t& d = descs_host[i];
@@ -2056,7 +2083,7 @@ int sasq_static_w8a8_linear_multi(int count, const sasq_linear_desc_t* descs_hos
             pp.a_int8 = reinterpret_cast<uint8_t*>(slice(i));
             pp.tile_begin = gp.num_tiles;
             pp.chunk_begin = gp.num_chunks;
-            if (!make_tmap(&maps.a[q], pp.a_int8, d.T, d.K, 128) ||
+            if (!make_tmap(&maps.a[q], pp.a_int8, d.T, d.K, small_layout ? P_SMALL_ROWS : 128) ||
                 !make_tmap(&maps.w[q], d.w, d.N, d.K, pp.w_box_rows) ||
                 !make_tmap_out(&maps.y64[q], d.y, d.T, d.N, 64) || !make_tmap_out(&maps.y16[q], d.y, d.T, d.N, 16))
                 return SASQ_ERR_CUDA;
@@ -2073,7 +2100,7 @@ int sasq_static_w8a8_linear_multi(int count, const sasq_linear_desc_t* descs_hos
         }
         gp.ready_count = off;
         deal_tiles_by_cost(&gp, pairs);
-        return launch_pair_group(maps, gp, pairs, bf, st);
+        return launch_pair_group(maps, gp, pairs, bf, st, small_layout);
     };
 
     return for_each_run(count, descs_host, pairs, [&](int first, int last, bool grouped) -> int {
