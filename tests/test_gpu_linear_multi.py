@@ -106,6 +106,18 @@ def test_small_t_problems_that_fill_the_chip_share_one_launch(tag):
     check_against_oracle(problems, tag)
 
 
+def test_single_row_block_problems_take_the_cost_dealt_tile_lists():
+    """Problems of up to 256 rows (one row block each) with different K: their tiles are dealt out by cost instead
+    of round-robin; with more than 32 rows the launch keeps the five-stage layout."""
+    tag = oracle.BF16
+    problems = [make_problem(200, 11008, 128, tag, 9800),
+                make_problem(256, 11008, 64, tag, 9810, with_bias=True),
+                make_problem(130, 4096, 320, tag, 9820),
+                make_problem(33, 4104, 48, tag, 9830)]
+    assert P.sasq_static_w8a8_linear_multi_launches([(pr["T"], pr["N"], pr["K"]) for pr in problems]) == 1
+    check_against_oracle(problems, tag)
+
+
 def test_llama7b_layer_at_decode_size_in_one_launch():
     """The seven linears of a LLaMA-2-7B layer at T = 16: one launch, every output row against the oracle for three
     of them, all seven bit-identical to separate calls (which take the small-T kernel)."""
