@@ -241,6 +241,24 @@ SASQ_API int sasq_static_w8a8_linear_per_channel(const void* x, const int8_t* w,
                                                  int32_t* acc_out, int64_t T, int64_t N, int64_t K, int dt, int bits,
                                                  void* workspace, size_t ws_bytes, void* stream);
 
+/* Bytes of scratch sasq_static_w8a8_linear_grouped needs for this shape. */
+SASQ_API size_t sasq_static_w8a8_linear_grouped_workspace(int64_t T, int64_t N, int64_t K);
+
+/* Static W8A8 linear in the grouped form of Eq. 3: the K axis is cut into K / group groups of `group` consecutive
+ * columns, each with its own static activation factor; a group's integer partial product is scaled by its factor
+ * and the partials are accumulated in fp32, in group order:
+ *   X_int[t,k] = int8(c(x[t,k])) with s = s_group[k / group]                       (Eq. 1 per group)
+ *   acc_g[t,n] = sum_{k in group g} X_int[t,k] * w[n,k]                            (int32)
+ *   y[t,n]     = narrow( sum_g fl32(acc_g) * fl32(s_group[g] * w_scale[n]) (+ bias[n]) )   (fp32 adds, g ascending,
+ *                                                                                   starting from +0, no FMA)
+ * s_group_dev: [K / group] fp32 in DEVICE memory.  group must be a multiple of 128 and divide K (otherwise
+ * SASQ_ERR_UNSUPPORTED).  Other arguments, alignment, ownership and errors as for sasq_static_w8a8_linear; there is
+ * no acc_out (no single integer accumulator exists).  Three launches: reciprocals, activation quantizer, GEMM. */
+SASQ_API int sasq_static_w8a8_linear_grouped(const void* x, const int8_t* w, const float* w_scale,
+                                             const float* s_group_dev, int64_t group, const void* bias, void* y,
+                                             int64_t T, int64_t N, int64_t K, int dt, int bits, void* workspace,
+                                             size_t ws_bytes, void* stream);
+
 /* Bytes of scratch sasq_dynamic_w8a8_linear needs for this shape. */
 SASQ_API size_t sasq_dynamic_w8a8_linear_workspace(int64_t T, int64_t N, int64_t K);
 

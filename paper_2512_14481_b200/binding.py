@@ -23,7 +23,8 @@ __all__ = [
     "sasq_fakequant_fwd_bwd_ablation", "sasq_adamw_scales", "SASQ_FULL_OPERATOR", "SASQ_WITHOUT_ROUND",
     "SASQ_WITHOUT_CLAMP", "sasq_dynamic_w8a8_linear_workspace", "sasq_dynamic_w8a8_linear", "sasq_debug_set_wait_limit", "PcDesc", "sasq_fakequant_per_channel_multi_workspace",
     "sasq_fakequant_fwd_bwd_per_channel_multi", "sasq_static_w8a8_linear_per_channel_workspace",
-    "sasq_static_w8a8_linear_per_channel", "LinearDesc", "sasq_static_w8a8_linear_multi_workspace",
+    "sasq_static_w8a8_linear_per_channel", "sasq_static_w8a8_linear_grouped_workspace",
+    "sasq_static_w8a8_linear_grouped", "LinearDesc", "sasq_static_w8a8_linear_multi_workspace",
     "sasq_static_w8a8_linear_multi", "sasq_static_w8a8_linear_multi_launches", "LinearProblems", "QuantTensors",
 ]
 
@@ -130,6 +131,10 @@ def load_library() -> ctypes.CDLL:
     L.sasq_fakequant_fwd_bwd_per_channel_multi.argtypes = [ctypes.POINTER(PcDesc), i32, i32, i32, i32, vp, sz, vp]
     L.sasq_debug_set_wait_limit.restype = ctypes.c_longlong
     L.sasq_debug_set_wait_limit.argtypes = [ctypes.c_longlong]
+    L.sasq_static_w8a8_linear_grouped_workspace.restype = sz
+    L.sasq_static_w8a8_linear_grouped_workspace.argtypes = [i64, i64, i64]
+    L.sasq_static_w8a8_linear_grouped.restype = i32
+    L.sasq_static_w8a8_linear_grouped.argtypes = [vp, vp, vp, vp, i64, vp, vp, i64, i64, i64, i32, i32, vp, sz, vp]
     L.sasq_static_w8a8_linear_multi_workspace.restype = sz
     L.sasq_static_w8a8_linear_multi_workspace.argtypes = [i32, ctypes.POINTER(LinearDesc)]
     L.sasq_static_w8a8_linear_multi.restype = i32
@@ -391,6 +396,33 @@ def sasq_static_w8a8_linear(x, w, w_scale, x_scale, y, bias=None, acc_out=None, 
     _check(load_library().sasq_static_w8a8_linear(_ptr(x), _ptr(w), _ptr(w_scale), _ptr(x_scale), _ptr(bias), _ptr(y),
                                                   _ptr(acc_out), T, N, K, _dt(x), int(bits), _ptr(workspace),
                                                   _nbytes(workspace), _stream(stream)), "sasq_static_w8a8_linear")
+
+
+def sasq_static_w8a8_linear_grouped_workspace(T: int, N: int, K: int) -> int:
+    return int(load_library().sasq_static_w8a8_linear_grouped_workspace(int(T), int(N), int(K)))
+
+
+def sasq_static_w8a8_linear_grouped(x, w, w_scale, s_group, group: int, y, bias=None, workspace=None, bits: int = 8,
+                                    stream=None) -> None:
+    """Eq. 3: x [T, K], one static factor per group of `group` consecutive channels (s_group [K / group])."""
+    _dev(x, "x"); _dev(w, "w", torch.int8); _dev(w_scale, "w_scale", torch.float32)
+    _dev(s_group, "s_group", torch.float32); _dev(y, "y", x.dtype)
+    if bias is not None:
+        _dev(bias, "bias", x.dtype)
+    if workspace is not None:
+        _dev(workspace, "workspace")
+    if x.dim() != 2 or w.dim() != 2 or x.shape[1] != w.shape[1]:
+        raise ValueError("x must be [T, K] and w [N, K]")
+    T, K = x.shape
+    N = w.shape[0]
+    if group <= 0 or K % group != 0 or s_group.numel() != K // group:
+        raise ValueError("s_group must hold one factor per group of `group` channels")
+    if tuple(y.shape) != (T, N) or w_scale.numel() != N or (bias is not None and bias.numel() != N):
+        raise ValueError("y must be [T, N], w_scale and bias [N]")
+    _check(load_library().sasq_static_w8a8_linear_grouped(_ptr(x), _ptr(w), _ptr(w_scale), _ptr(s_group), int(group),
+                                                          _ptr(bias), _ptr(y), T, N, K, _dt(x), int(bits),
+                                                          _ptr(workspace), _nbytes(workspace), _stream(stream)),
+           "sasq_static_w8a8_linear_grouped")
 
 
 def _linear_descs(problems):

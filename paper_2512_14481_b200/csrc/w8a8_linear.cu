@@ -305,6 +305,243 @@ w8a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 
 
 // ---------------------------------------------------------------------------
+// Grouped form (Eq. 3): K is cut into groups of `group` columns, each with its own activation factor s_g.  The
+// integer partial product of a group cannot be carried into the next one, so every group gets a fresh int32
+// accumulator in TMEM (two of them, alternating), and the epilogue warps fold it into an fp32 running sum that also
+// lives in TMEM (read, v + fl32(acc) * fl32(s_g * s_w[n]), written back) while the MMAs of the next group run:
+//   y[t,n] = narrow( sum_g fl32(acc_g[t,n]) * fl32(s_g * s_w[n]) (+ bias[n]) ),   groups in order, fp32, no FMA.
+// One CTA per 128 x 128 tile; TMEM columns [0,128) and [128,256) int32, [256,384) the fp32 sums.
+// ---------------------------------------------------------------------------
+constexpr int GBN = 128;
+constexpr int G_STAGE_BYTES = BM * BK + GBN * BK;            // 32 KB
+constexpr int G_STAGES = (STAGES * STAGE_BYTES) / G_STAGE_BYTES;   // the same ring: 6 stages
+static_assert(G_STAGES <= 8, "GroupedTail holds the barriers of up to 8 stages");
+
+struct GroupedTail {
+    uint64_t full[8];
+    uint64_t empty[8];
+    uint64_t tmem_full[ACC_BUFS];
+    uint64_t tmem_empty[ACC_BUFS];
+    float scale[GBN];              // s_w[n] of the tile's columns
+    float bias[GBN];
+    uint32_t tmem_base;
+    volatile int abort_flag;
+};
+
+constexpr size_t kGroupedSmemBytes = 1024 /* alignment slack */ + (size_t)G_STAGES * G_STAGE_BYTES + sizeof(GroupedTail);
+
+struct GroupedParams {
+    LinearParams lp;               // x_scale, row_scale, chan_inv unused here
+    const float* s_group;          // [groups] activation factor of each K group
+    int group_kblocks;             // k-blocks (of 128 columns) per group
+    int groups;
+};
+
+__device__ __forceinline__ bool wait_bounded_g(uint64_t* bar, uint32_t parity, GroupedTail* tail, const LinearParams& p) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    int polls = 0;
+    while (!ptx::mbar_try_wait(bar, parity)) {
+        if (p.wait_limit <= 0 || (++polls & 63) == 0) {
+            if (tail->abort_flag) return false;
+            if (clock64() - t0 > p.wait_limit) {
+                tail->abort_flag = 1;
+                atomicMax(p.status, (int)SASQ_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+template <bool BF>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+w8a8_grouped_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
+                    const __grid_constant__ GroupedParams gp) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    GroupedTail* tail = reinterpret_cast<GroupedTail*>(tiles + (size_t)G_STAGES * G_STAGE_BYTES);
+    const LinearParams& p = gp.lp;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < G_STAGES; ++s) {
+            ptx::mbar_init(&tail->full[s], 1);
+            ptx::mbar_init(&tail->empty[s], 1);
+        }
+        for (int b = 0; b < ACC_BUFS; ++b) {
+            ptx::mbar_init(&tail->tmem_full[b], 1);
+            ptx::mbar_init(&tail->tmem_empty[b], EPI_THREADS);
+        }
+        tail->abort_flag = 0;
+        ptx::mbar_init_fence();
+        ptx::prefetch_tensormap(&tmap_a);
+        ptx::prefetch_tensormap(&tmap_w);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(&tail->tmem_base, TMEM_COLS);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = tail->tmem_base;
+
+    const int num_tiles = p.m_blocks * p.n_blocks;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (ptx::elect_one()) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                const int m_blk = tile % p.m_blocks, n_blk = tile / p.m_blocks;
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    ok = wait_bounded_g(&tail->empty[stage], phase ^ 1u, tail, p);
+                    if (!ok) break;
+                    uint8_t* a_dst = tiles + (size_t)stage * G_STAGE_BYTES;
+                    uint8_t* b_dst = a_dst + BM * BK;
+                    ptx::mbar_arrive_expect_tx(&tail->full[stage], G_STAGE_BYTES);
+                    ptx::tma_load_2d(a_dst, &tmap_a, &tail->full[stage], kb * BK, m_blk * BM);
+                    ptx::tma_load_2d(b_dst, &tmap_w, &tail->full[stage], kb * BK, n_blk * GBN);
+                    if (++stage == G_STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+            // after an abort, copies still in flight must land before the CTA's shared memory goes away
+            if (!ok) {
+                for (int s = 0; s < G_STAGES; ++s) {
+                    const long long t0 = clock64();
+                    const uint32_t par = (s < stage) ? phase : (phase ^ 1u);
+                    while (!ptx::mbar_try_wait(&tail->full[s], par)) {
+                        if (clock64() - t0 > (1LL << 24)) break;
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ---------------- MMA issuer: a fresh accumulator for every group ----------------
+        if (ptx::elect_one()) {
+            constexpr uint32_t idesc = ptx::idesc_i8(BM, GBN);
+            const uint64_t a_desc0 = ptx::smem_desc_k_major_sw128(ptx::smem_u32(tiles));
+            const uint64_t b_desc0 = ptx::smem_desc_k_major_sw128(ptx::smem_u32(tiles) + BM * BK);
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            int it = 0;                 // groups issued so far by this CTA
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                for (int g = 0; g < gp.groups && ok; ++g, ++it) {
+                    const int buf = it & 1;
+                    const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+                    ok = wait_bounded_g(&tail->tmem_empty[buf], acc_phase ^ 1u, tail, p);
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
+                    const uint32_t d_tmem = tmem_base + (uint32_t)(buf * GBN);
+                    uint32_t accumulate = 0;
+                    for (int kb = 0; kb < gp.group_kblocks; ++kb) {
+                        ok = wait_bounded_g(&tail->full[stage], phase, tail, p);
+                        if (!ok) break;
+                        ptx::tc_fence_after_sync();
+                        const uint64_t a_desc = a_desc0 + (uint64_t)(stage * (G_STAGE_BYTES >> 4));
+                        const uint64_t b_desc = b_desc0 + (uint64_t)(stage * (G_STAGE_BYTES >> 4));
+                        ptx::mma_i8_ss(d_tmem, a_desc, b_desc, idesc, accumulate);
+                        ptx::mma_i8_ss_acc(d_tmem, a_desc + 2, b_desc + 2, idesc);
+                        ptx::mma_i8_ss_acc(d_tmem, a_desc + 4, b_desc + 4, idesc);
+                        ptx::mma_i8_ss_acc(d_tmem, a_desc + 6, b_desc + 6, idesc);
+                        accumulate = 1u;
+                        ptx::mma_commit(&tail->empty[stage]);
+                        if (kb == gp.group_kblocks - 1) ptx::mma_commit(&tail->tmem_full[buf]);
+                        if (++stage == G_STAGES) { stage = 0; phase ^= 1u; }
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else {
+        // ---------------- epilogue (warps 2..5): fold each group into the fp32 sums ----------------
+        const int quad = warp & 3;
+        const int et = threadIdx.x - 64;
+        const bool has_bias = p.bias != nullptr;
+        bool ok = true;
+        int it = 0;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            const int m_blk = tile % p.m_blocks, n_blk = tile / p.m_blocks;
+            const int n0 = n_blk * GBN;
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            for (int j = et; j < GBN; j += EPI_THREADS) {
+                const int n = n0 + j;
+                tail->scale[j] = (n < p.N) ? __ldg(p.w_scale + n) : 0.0f;
+                if (has_bias)
+                    tail->bias[j] = (n < p.N) ? widen1<BF>(__ldg(reinterpret_cast<const uint16_t*>(p.bias) + n)) : 0.0f;
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            const int row = m_blk * BM + quad * 32 + lane;
+            const bool row_ok = row < p.T;
+            uint16_t* yrow = reinterpret_cast<uint16_t*>(p.y) + (size_t)row * p.N + n0;
+            const uint32_t lanes = tmem_base + ((uint32_t)(quad * 32) << 16);
+            for (int g = 0; g < gp.groups && ok; ++g, ++it) {
+                const int buf = it & 1;
+                const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+                const float sg = __ldg(gp.s_group + g);
+                if (tile == 0 && et == 0 && scale_is_bad(sg)) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
+                ok = wait_bounded_g(&tail->tmem_full[buf], acc_phase, tail, p);
+                ok = epilogue_all_ok(ok);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                const bool first = g == 0, last = g == gp.groups - 1;
+#pragma unroll 1
+                for (int c = 0; c < GBN; c += 32) {
+                    uint32_t a[32], v[32];
+                    ptx::tmem_ld_32x32(lanes + (uint32_t)(buf * GBN + c), a);
+                    if (!first) ptx::tmem_ld_32x32(lanes + (uint32_t)(2 * GBN + c), v);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const float run = first ? 0.0f : __uint_as_float(v[j]);
+                        const float term = __fmul_rn(__int2float_rn((int)a[j]), __fmul_rn(sg, tail->scale[c + j]));
+                        v[j] = __float_as_uint(__fadd_rn(run, term));
+                    }
+                    if (!last) {
+                        ptx::tmem_st_32x32(lanes + (uint32_t)(2 * GBN + c), v);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8) {
+                            if (row_ok && (n0 + c + j) < p.N) {       // N % 8 == 0: eight columns are in or out together
+                                uint32_t o[4];
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    float f0 = __uint_as_float(v[j + 2 * q]), f1 = __uint_as_float(v[j + 2 * q + 1]);
+                                    if (has_bias) {
+                                        f0 = __fadd_rn(f0, tail->bias[c + j + 2 * q]);
+                                        f1 = __fadd_rn(f1, tail->bias[c + j + 2 * q + 1]);
+                                    }
+                                    o[q] = narrow2<BF>(f0, f1);
+                                }
+                                *reinterpret_cast<uint4*>(yrow + c + j) = make_uint4(o[0], o[1], o[2], o[3]);
+                            }
+                        }
+                    }
+                }
+                if (!last) ptx::tmem_st_wait();        // the sums are in TMEM before this warp reads them again
+                ptx::tc_fence_before_sync();
+                ptx::mbar_arrive(&tail->tmem_empty[buf]);
+            }
+        }
+    }
+
+    // ---------------- teardown ----------------
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ---------------------------------------------------------------------------
 // CTA-pair kernel (cta_group::2): two CTAs on neighbouring SMs share one 256 x BN
 // output tile.  CTA r of the pair keeps rows [128 r, 128 r + 128) of A and rows
 // [BN/2 r, BN/2 (r+1)) of W in its own shared memory, so each byte of W is read
@@ -1327,14 +1564,15 @@ __global__ void __launch_bounds__(256) quantize_act_kernel(const uint4* __restri
                                      : quantize8_channels<BF>(x[i], chan_inv + 8 * (unsigned)(i % vec_per_row), qn, qp);
 }
 
-// reciprocals of the per-channel factors, fl32(1 / s[k]), once per call; a zero / non-finite factor is reported
+// reciprocals of the per-channel factors, fl32(1 / s[k / group]) (group = 1: one factor per channel), once per
+// call; a zero / non-finite factor is reported
 __global__ void __launch_bounds__(256) reciprocal_factors_kernel(const float* __restrict__ s, float* __restrict__ inv,
-                                                                 int K, int* status) {
+                                                                 int K, int group, int* status) {
     pdl_launch_dependents();
     pdl_wait();
     const int k = blockIdx.x * 256 + threadIdx.x;
     if (k >= K) return;
-    const float sk = s[k];
+    const float sk = s[k / group];
     if (scale_is_bad(sk)) atomicMax(status, (int)SASQ_ERR_BAD_SCALE);
     inv[k] = __fdiv_rn(1.0f, sk);
 }
@@ -1851,7 +2089,7 @@ int linear_impl(const void* x, const int8_t* w, const float* w_scale, const floa
         cudaLaunchAttribute attr[1] = {pdl_attribute()};
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, reciprocal_factors_kernel, x_scales_vec, inv, (int)K, status) != cudaSuccess)
+        if (cudaLaunchKernelEx(&cfg, reciprocal_factors_kernel, x_scales_vec, inv, (int)K, 1, status) != cudaSuccess)
             return SASQ_ERR_CUDA;
         chan_inv = inv;
     }
@@ -2134,6 +2372,87 @@ int sasq_static_w8a8_linear_multi_launches(int count, const sasq_linear_desc_t* 
         return SASQ_OK;
     });
     return launches;
+}
+
+size_t sasq_static_w8a8_linear_grouped_workspace(int64_t T, int64_t N, int64_t K) {
+    (void)N;
+    if (T <= 0 || K <= 0) return 0;
+    // int8 codes, then one fp32 reciprocal per channel (the group's, repeated)
+    return sasq_static_w8a8_linear_workspace(T, N, K) + 256 + (size_t)K * sizeof(float) + 256;
+}
+
+int sasq_static_w8a8_linear_grouped(const void* x, const int8_t* w, const float* w_scale, const float* s_group_dev,
+                                    int64_t group, const void* bias, void* y, int64_t T, int64_t N, int64_t K, int dt,
+                                    int bits, void* workspace, size_t ws_bytes, void* stream) {
+    using namespace sasq;
+    if (s_group_dev == nullptr || group <= 0) return SASQ_ERR_INVALID_ARG;
+    const int rc = check_linear_args(x, w, w_scale, nullptr, s_group_dev, false, nullptr, bias, y, nullptr, T, N, K, dt,
+                                     bits);
+    if (rc != SASQ_OK) return rc;
+    if (group % BK != 0 || K % group != 0) return SASQ_ERR_UNSUPPORTED;      // groups are whole 128-column k-blocks
+    if (T == 0) return SASQ_OK;
+    if (workspace == nullptr || !aligned16(workspace) || ws_bytes < sasq_static_w8a8_linear_grouped_workspace(T, N, K))
+        return SASQ_ERR_WORKSPACE;
+    const int sm_count = device_sm_count_if_sm100();
+    if (sm_count <= 0) return SASQ_ERR_UNSUPPORTED;
+    int* status = status_word_ptr();
+    if (status == nullptr) return SASQ_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool bf = dt == SASQ_BF16;
+    {
+        static bool ready[64][2] = {};
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SASQ_ERR_CUDA;
+        if (!ready[dev][bf]) {
+            const void* fn = bf ? reinterpret_cast<const void*>(w8a8_grouped_kernel<true>)
+                                : reinterpret_cast<const void*>(w8a8_grouped_kernel<false>);
+            if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGroupedSmemBytes) !=
+                cudaSuccess)
+                return SASQ_ERR_CUDA;
+            ready[dev][bf] = true;
+        }
+    }
+    uint8_t* a_int8 = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(workspace) + 127) & ~uintptr_t(127));
+    float* inv = reinterpret_cast<float*>(reinterpret_cast<uintptr_t>(a_int8) + (uintptr_t)((T * K + 255) / 256 * 256));
+    const float qn = (float)(1 << (bits - 1)), qp = (float)((1 << (bits - 1)) - 1);
+
+    // 1. fl32(1 / s_g) for every channel of its group, 2. Eq. 1 with those -> int8 codes, 3. the grouped GEMM
+    reciprocal_factors_kernel<<<(unsigned)((K + 255) / 256), 256, 0, st>>>(s_group_dev, inv, (int)K, (int)group, status);
+    const long long n8 = (T * K) / 8;
+    long long blocks = (n8 + 255) / 256;
+    if (blocks > (long long)sm_count * 8) blocks = (long long)sm_count * 8;
+    if (bf)
+        quantize_act_kernel<true><<<(int)blocks, 256, 0, st>>>(static_cast<const uint4*>(x),
+                                                               reinterpret_cast<uint2*>(a_int8), n8, nullptr, inv,
+                                                               (unsigned)(K / 8), qn, qp);
+    else
+        quantize_act_kernel<false><<<(int)blocks, 256, 0, st>>>(static_cast<const uint4*>(x),
+                                                                reinterpret_cast<uint2*>(a_int8), n8, nullptr, inv,
+                                                                (unsigned)(K / 8), qn, qp);
+    if (cudaGetLastError() != cudaSuccess) return SASQ_ERR_CUDA;
+
+    GroupedParams gp{};
+    LinearParams& p = gp.lp;
+    p.w_scale = w_scale;
+    p.bias = bias;
+    p.y = y;
+    p.T = (int)T; p.N = (int)N; p.K = (int)K;
+    p.k_blocks = (int)(K / BK);
+    p.m_blocks = (int)((T + BM - 1) / BM);
+    p.n_blocks = (int)((N + GBN - 1) / GBN);
+    p.status = status;
+    p.wait_limit = g_wait_limit.load(std::memory_order_relaxed);
+    gp.s_group = s_group_dev;
+    gp.group_kblocks = (int)(group / BK);
+    gp.groups = (int)(K / group);
+    CUtensorMap tmap_a, tmap_w;
+    if (!make_tmap(&tmap_a, a_int8, T, K, BM) || !make_tmap(&tmap_w, w, N, K, GBN)) return SASQ_ERR_CUDA;
+    const long long tiles = (long long)p.m_blocks * p.n_blocks;
+    const int grid = (int)(tiles < sm_count ? tiles : sm_count);
+    if (bf) w8a8_grouped_kernel<true><<<grid, NUM_THREADS, kGroupedSmemBytes, st>>>(tmap_a, tmap_w, gp);
+    else w8a8_grouped_kernel<false><<<grid, NUM_THREADS, kGroupedSmemBytes, st>>>(tmap_a, tmap_w, gp);
+    if (cudaGetLastError() != cudaSuccess) return SASQ_ERR_CUDA;
+    return SASQ_OK;
 }
 
 size_t sasq_static_w8a8_linear_per_channel_workspace(int64_t T, int64_t N, int64_t K) {
