@@ -307,15 +307,19 @@ w8a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 // ---------------------------------------------------------------------------
 // Grouped form (Eq. 3): K is cut into groups of `group` columns, each with its own activation factor s_g.  The
 // integer partial product of a group cannot be carried into the next one, so every group gets a fresh int32
-// accumulator in TMEM (two of them, alternating), and the epilogue warps fold it into an fp32 running sum that also
-// lives in TMEM (read, v + fl32(acc) * fl32(s_g * s_w[n]), written back) while the MMAs of the next group run:
+// accumulator in TMEM (two of them, alternating), and while the MMAs of the next group run the folding warps add it
+// to fp32 running sums that they keep in registers (v + fl32(acc) * fl32(s_g * s_w[n])):
 //   y[t,n] = narrow( sum_g fl32(acc_g[t,n]) * fl32(s_g * s_w[n]) (+ bias[n]) ),   groups in order, fp32, no FMA.
-// One CTA per 128 x 128 tile; TMEM columns [0,128) and [128,256) int32, [256,384) the fp32 sums.
+// One CTA per 128 x 128 tile; TMEM columns [0,128) and [128,256) hold the two int32 accumulators.  With small groups
+// the folding, not the MMAs, sets the pace (a 128-column group is four MMAs), so eight warps do it: two per TMEM
+// lane quadrant, 64 columns (64 sums per thread) each.
 // ---------------------------------------------------------------------------
 constexpr int GBN = 128;
 constexpr int G_STAGE_BYTES = BM * BK + GBN * BK;            // 32 KB
 constexpr int G_STAGES = (STAGES * STAGE_BYTES) / G_STAGE_BYTES;   // the same ring: 6 stages
 static_assert(G_STAGES <= 8, "GroupedTail holds the barriers of up to 8 stages");
+constexpr int G_EPI_THREADS = 256;
+constexpr int G_THREADS = 64 + G_EPI_THREADS;
 
 struct GroupedTail {
     uint64_t full[8];
@@ -354,8 +358,24 @@ __device__ __forceinline__ bool wait_bounded_g(uint64_t* bar, uint32_t parity, G
     return true;
 }
 
+// Barrier over the 256 folding threads (named barrier 2) that also ANDs a predicate.
+__device__ __forceinline__ bool grouped_all_ok(bool ok) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p, q;\n\t"
+        "setp.ne.b32 q, %1, 0;\n\t"
+        "bar.red.and.pred p, 2, 256, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}"
+        : "=r"(r)
+        : "r"((uint32_t)ok)
+        : "memory");
+    return r != 0;
+}
+
 template <bool BF>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(G_THREADS, 1)
 w8a8_grouped_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                     const __grid_constant__ GroupedParams gp) {
     extern __shared__ uint8_t smem_raw[];
@@ -373,7 +393,7 @@ w8a8_grouped_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         }
         for (int b = 0; b < ACC_BUFS; ++b) {
             ptx::mbar_init(&tail->tmem_full[b], 1);
-            ptx::mbar_init(&tail->tmem_empty[b], EPI_THREADS);
+            ptx::mbar_init(&tail->tmem_empty[b], G_EPI_THREADS / 32);       // one arrival per folding warp
         }
         tail->abort_flag = 0;
         ptx::mbar_init_fence();
@@ -461,8 +481,9 @@ w8a8_grouped_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         }
         __syncwarp();
     } else {
-        // ---------------- epilogue (warps 2..5): fold each group into the fp32 sums ----------------
-        const int quad = warp & 3;
+        // ---------------- warps 2..9: fold each group into the fp32 sums ----------------
+        const int quad = warp & 3;                      // TMEM lane quadrant this warp may access
+        const int c_begin = warp < 6 ? 0 : GBN / 2;     // its half of the tile's columns
         const int et = threadIdx.x - 64;
         const bool has_bias = p.bias != nullptr;
         bool ok = true;
@@ -470,65 +491,65 @@ w8a8_grouped_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
             const int m_blk = tile % p.m_blocks, n_blk = tile / p.m_blocks;
             const int n0 = n_blk * GBN;
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            for (int j = et; j < GBN; j += EPI_THREADS) {
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            for (int j = et; j < GBN; j += G_EPI_THREADS) {
                 const int n = n0 + j;
                 tail->scale[j] = (n < p.N) ? __ldg(p.w_scale + n) : 0.0f;
                 if (has_bias)
                     tail->bias[j] = (n < p.N) ? widen1<BF>(__ldg(reinterpret_cast<const uint16_t*>(p.bias) + n)) : 0.0f;
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            asm volatile("bar.sync 1, 256;" ::: "memory");
             const int row = m_blk * BM + quad * 32 + lane;
             const bool row_ok = row < p.T;
             uint16_t* yrow = reinterpret_cast<uint16_t*>(p.y) + (size_t)row * p.N + n0;
             const uint32_t lanes = tmem_base + ((uint32_t)(quad * 32) << 16);
+            float run[GBN / 2];                         // the sums of this thread's row; +0 to start with
+#pragma unroll
+            for (int j = 0; j < GBN / 2; ++j) run[j] = 0.0f;
             for (int g = 0; g < gp.groups && ok; ++g, ++it) {
                 const int buf = it & 1;
                 const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
                 const float sg = __ldg(gp.s_group + g);
                 if (tile == 0 && et == 0 && scale_is_bad(sg)) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
+                // every warp waits on its own: whoever gives up raises the abort flag, which ends the others' waits
                 ok = wait_bounded_g(&tail->tmem_full[buf], acc_phase, tail, p);
-                ok = epilogue_all_ok(ok);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-                const bool first = g == 0, last = g == gp.groups - 1;
-#pragma unroll 1
-                for (int c = 0; c < GBN; c += 32) {
-                    uint32_t a[32], v[32];
-                    ptx::tmem_ld_32x32(lanes + (uint32_t)(buf * GBN + c), a);
-                    if (!first) ptx::tmem_ld_32x32(lanes + (uint32_t)(2 * GBN + c), v);
-                    ptx::tmem_ld_wait();
+                uint32_t a0[32], a1[32];
+                ptx::tmem_ld_32x32(lanes + (uint32_t)(buf * GBN + c_begin), a0);
+                ptx::tmem_ld_32x32(lanes + (uint32_t)(buf * GBN + c_begin + 32), a1);
+                ptx::tmem_ld_wait();
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const float run = first ? 0.0f : __uint_as_float(v[j]);
-                        const float term = __fmul_rn(__int2float_rn((int)a[j]), __fmul_rn(sg, tail->scale[c + j]));
-                        v[j] = __float_as_uint(__fadd_rn(run, term));
-                    }
-                    if (!last) {
-                        ptx::tmem_st_32x32(lanes + (uint32_t)(2 * GBN + c), v);
-                    } else {
+                for (int j = 0; j < 32; ++j) {
+                    run[j] = __fadd_rn(run[j], __fmul_rn(__int2float_rn((int)a0[j]),
+                                                         __fmul_rn(sg, tail->scale[c_begin + j])));
+                    run[32 + j] = __fadd_rn(run[32 + j], __fmul_rn(__int2float_rn((int)a1[j]),
+                                                                   __fmul_rn(sg, tail->scale[c_begin + 32 + j])));
+                }
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&tail->tmem_empty[buf]);
+            }
+            if (ok && row_ok) {
 #pragma unroll
-                        for (int j = 0; j < 32; j += 8) {
-                            if (row_ok && (n0 + c + j) < p.N) {       // N % 8 == 0: eight columns are in or out together
-                                uint32_t o[4];
+                for (int j = 0; j < GBN / 2; j += 8) {
+                    if (n0 + c_begin + j < p.N) {               // N % 8 == 0: eight columns are in or out together
+                        uint32_t o[4];
 #pragma unroll
-                                for (int q = 0; q < 4; ++q) {
-                                    float f0 = __uint_as_float(v[j + 2 * q]), f1 = __uint_as_float(v[j + 2 * q + 1]);
-                                    if (has_bias) {
-                                        f0 = __fadd_rn(f0, tail->bias[c + j + 2 * q]);
-                                        f1 = __fadd_rn(f1, tail->bias[c + j + 2 * q + 1]);
-                                    }
-                                    o[q] = narrow2<BF>(f0, f1);
-                                }
-                                *reinterpret_cast<uint4*>(yrow + c + j) = make_uint4(o[0], o[1], o[2], o[3]);
+                        for (int q = 0; q < 4; ++q) {
+                            float f0 = run[j + 2 * q], f1 = run[j + 2 * q + 1];
+                            if (has_bias) {
+                                f0 = __fadd_rn(f0, tail->bias[c_begin + j + 2 * q]);
+                                f1 = __fadd_rn(f1, tail->bias[c_begin + j + 2 * q + 1]);
                             }
+                            o[q] = narrow2<BF>(f0, f1);
                         }
+                        *reinterpret_cast<uint4*>(yrow + c_begin + j) = make_uint4(o[0], o[1], o[2], o[3]);
                     }
                 }
-                if (!last) ptx::tmem_st_wait();        // the sums are in TMEM before this warp reads them again
-                ptx::tc_fence_before_sync();
-                ptx::mbar_arrive(&tail->tmem_empty[buf]);
             }
+            // the 256 threads go on to the next tile's barrier together or leave together
+            ok = grouped_all_ok(ok);
         }
     }
 
@@ -2449,8 +2470,8 @@ int sasq_static_w8a8_linear_grouped(const void* x, const int8_t* w, const float*
     if (!make_tmap(&tmap_a, a_int8, T, K, BM) || !make_tmap(&tmap_w, w, N, K, GBN)) return SASQ_ERR_CUDA;
     const long long tiles = (long long)p.m_blocks * p.n_blocks;
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
-    if (bf) w8a8_grouped_kernel<true><<<grid, NUM_THREADS, kGroupedSmemBytes, st>>>(tmap_a, tmap_w, gp);
-    else w8a8_grouped_kernel<false><<<grid, NUM_THREADS, kGroupedSmemBytes, st>>>(tmap_a, tmap_w, gp);
+    if (bf) w8a8_grouped_kernel<true><<<grid, G_THREADS, kGroupedSmemBytes, st>>>(tmap_a, tmap_w, gp);
+    else w8a8_grouped_kernel<false><<<grid, G_THREADS, kGroupedSmemBytes, st>>>(tmap_a, tmap_w, gp);
     if (cudaGetLastError() != cudaSuccess) return SASQ_ERR_CUDA;
     return SASQ_OK;
 }
