@@ -350,6 +350,18 @@ SASQ_API int sasq_adamw_scales(float* scales_dev, const float* grad_scales_dev, 
                                float* exp_avg_sq_dev, int n, int step, float lr, float beta1, float beta2, float eps,
                                float weight_decay, void* stream);
 
+/* Concurrency of the linear entry points.  When the activation quantizer runs inside the GEMM launch (every static
+ * linear with T <= 262144 whose tiles fit the device), CTAs of that launch wait for codes that other CTAs of the
+ * same launch write, so the launch is sized to be resident as a whole -- on an otherwise free device.  If kernels on
+ * OTHER streams hold SMs meanwhile, the missing CTAs start when those kernels end; two such launches that overlap on
+ * different streams can each hold the SMs the other is waiting for, in which case their bounded waits give up after
+ * about a second with SASQ_ERR_TIMEOUT (outputs unspecified, nothing hangs).  Callers that run these entry points
+ * on several streams of one device at once, or beside long-running kernels, switch this on: the launches are then
+ * made as co-operative grids, which the driver starts only when every CTA can be resident.  It costs the overlap of
+ * a launch's set-up with its predecessor's tail, about 2 us per launch on a B200.  on: non-zero / zero; applies to
+ * launches made afterwards, process-wide; returns the previous setting (default 0).  The paper has no counterpart. */
+SASQ_API int sasq_set_gang_launch(int on);
+
 /* Test hook.  Every wait inside the GEMM kernels (on an mbarrier, on the activation quantizer's counters) gives up
  * after this many SM clock cycles, raises SASQ_ERR_TIMEOUT in the status word and lets the kernel finish in an
  * orderly way (outputs are then unspecified).  The default is 2^31 cycles, about a second; a negative value restores

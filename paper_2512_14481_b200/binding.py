@@ -25,7 +25,7 @@ __all__ = [
     "sasq_fakequant_fwd_bwd_per_channel_multi", "sasq_static_w8a8_linear_per_channel_workspace",
     "sasq_static_w8a8_linear_per_channel", "sasq_static_w8a8_linear_grouped_workspace",
     "sasq_static_w8a8_linear_grouped", "LinearDesc", "sasq_static_w8a8_linear_multi_workspace",
-    "sasq_static_w8a8_linear_multi", "sasq_static_w8a8_linear_multi_launches", "LinearProblems", "QuantTensors",
+    "sasq_static_w8a8_linear_multi", "sasq_static_w8a8_linear_multi_launches", "sasq_set_gang_launch", "LinearProblems", "QuantTensors",
 ]
 
 SASQ_F16 = 0
@@ -563,6 +563,15 @@ def sasq_static_w8a8_linear_tiles(T: int, N: int, num_pairs: int, pair_id: int):
 def sasq_debug_set_wait_limit(cycles: int) -> int:
     """Test hook: clock cycles after which a wait inside the GEMM kernels gives up (negative restores the default)."""
     return int(load_library().sasq_debug_set_wait_limit(int(cycles)))
+
+
+def sasq_set_gang_launch(on: bool) -> bool:
+    """Launch the linears whose CTAs wait on one another as co-operative grids (for callers that overlap them on
+    several streams); returns the previous setting."""
+    L = load_library()
+    L.sasq_set_gang_launch.restype = ctypes.c_int
+    L.sasq_set_gang_launch.argtypes = [ctypes.c_int]
+    return bool(L.sasq_set_gang_launch(1 if on else 0))
 
 
 def sasq_device_status(stream=None) -> int:

@@ -47,6 +47,7 @@ constexpr int EPI_THREADS = 128;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr long long kWaitLimit = 1LL << 31;   // clock cycles a single wait may take (about a second)
 std::atomic<long long> g_wait_limit{kWaitLimit};   // what launches use; tests shorten it to see the give-up path
+std::atomic<int> g_gang_launch{0};                 // launch the kernels whose CTAs wait on one another as co-operative grids
 
 struct SharedTail {
     uint64_t full[STAGES];
@@ -1883,6 +1884,10 @@ bool single_kernel_ready(bool bf) {
 
 extern "C" {
 
+int sasq_set_gang_launch(int on) {
+    return sasq::g_gang_launch.exchange(on ? 1 : 0, std::memory_order_relaxed);
+}
+
 long long sasq_debug_set_wait_limit(long long cycles) {
     const long long want = cycles < 0 ? sasq::kWaitLimit : cycles;
     return sasq::g_wait_limit.exchange(want, std::memory_order_relaxed);
@@ -2007,14 +2012,16 @@ int launch_pair_group(const GroupMaps& maps, const GroupParams& gp, int pairs, b
     cfg.blockDim = dim3(P_NUM_THREADS, 1, 1);
     cfg.dynamicSmemBytes = kPairSmemBytes;
     cfg.stream = st;
-    cudaLaunchAttribute attr[2];
+    cudaLaunchAttribute attr[3];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     attr[1] = pdl_attribute();
+    attr[2].id = cudaLaunchAttributeCooperative;
+    attr[2].val.cooperative = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 2;
+    cfg.numAttrs = (gp.num_chunks != 0 && g_gang_launch.load(std::memory_order_relaxed)) ? 3 : 2;
     cudaError_t e;
     if (small_layout) {
         if (bf) e = cudaLaunchKernelEx(&cfg, w8a8_gemm_pair_kernel<true, true>, maps, gp);
@@ -2196,14 +2203,16 @@ int linear_impl(const void* x, const int8_t* w, const float* w_scale, const floa
         cfg.blockDim = dim3(D_THREADS, 1, 1);
         cfg.dynamicSmemBytes = kDecodeSmem;
         cfg.stream = st;
-        cudaLaunchAttribute attr[2];
+        cudaLaunchAttribute attr[3];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = (unsigned)split;
         attr[0].val.clusterDim.y = 1;
         attr[0].val.clusterDim.z = 1;
         attr[1] = pdl_attribute();
+        attr[2].id = cudaLaunchAttributeCooperative;
+        attr[2].val.cooperative = 1;
         cfg.attrs = attr;
-        cfg.numAttrs = 2;
+        cfg.numAttrs = (dp.x != nullptr && g_gang_launch.load(std::memory_order_relaxed)) ? 3 : 2;
         if (dt == SASQ_BF16) e = cudaLaunchKernelEx(&cfg, w8a8_decode_kernel<true>, tmap_w, tmap_a, dp);
         else e = cudaLaunchKernelEx(&cfg, w8a8_decode_kernel<false>, tmap_w, tmap_a, dp);
         if (e != cudaSuccess) return SASQ_ERR_CUDA;
