@@ -41,3 +41,45 @@ def test_a_wait_that_runs_out_is_reported_and_the_next_call_is_clean(T):
     xb = oracle.bits_of(x[idx].cpu())[0]
     y_o, _, _ = oracle.w8a8_linear(xb, tag, w_int.cpu().numpy(), w_scale.cpu().numpy(), 0.05, 8)
     assert np.array_equal(oracle.bits_of(y[idx].cpu())[0], y_o)
+
+
+def test_give_up_path_of_a_multi_problem_launch_and_of_the_grouped_form():
+    """The same for a launch that carries several problems and for the grouped (Eq. 3) kernel: the wait runs out,
+    the status word says so, and the next call with the default limit matches an untouched reference run."""
+    dev = torch.device("cuda")
+    shapes = [(300, 520, 512), (700, 264, 1024)]
+    probs = []
+    for i, (T, N, K) in enumerate(shapes):
+        probs.append((W.activations(T, K, torch.bfloat16, 9950 + i, device=dev),
+                      torch.randint(-127, 128, (N, K), dtype=torch.int8, device=dev),
+                      torch.full((N,), 1e-3, device=dev), torch.tensor([0.05], device=dev),
+                      torch.empty((T, N), dtype=torch.bfloat16, device=dev)))
+    ws = torch.empty(P.sasq_static_w8a8_linear_multi_workspace(shapes), dtype=torch.uint8, device=dev)
+    T, N, K, group = 300, 264, 1024, 256
+    xg = W.activations(T, K, torch.bfloat16, 9960, device=dev)
+    wg = torch.randint(-127, 128, (N, K), dtype=torch.int8, device=dev)
+    wsg = torch.full((N,), 1e-3, device=dev)
+    sg = torch.full((K // group,), 0.05, device=dev)
+    yg = torch.empty((T, N), dtype=torch.bfloat16, device=dev)
+    wsp = torch.empty(P.sasq_static_w8a8_linear_grouped_workspace(T, N, K), dtype=torch.uint8, device=dev)
+
+    def run_all():
+        P.sasq_static_w8a8_linear_multi(probs, ws)
+        P.sasq_static_w8a8_linear_grouped(xg, wg, wsg, sg, group, yg, workspace=wsp)
+
+    run_all()
+    assert P.sasq_device_status() == 0
+    want = [pr[4].clone() for pr in probs] + [yg.clone()]
+    for call in (lambda: P.sasq_static_w8a8_linear_multi(probs, ws),
+                 lambda: P.sasq_static_w8a8_linear_grouped(xg, wg, wsg, sg, group, yg, workspace=wsp)):
+        P.sasq_debug_set_wait_limit(0)
+        try:
+            call()
+            status = P.sasq_device_status()
+        finally:
+            P.sasq_debug_set_wait_limit(-1)
+        assert status == SASQ_ERR_TIMEOUT
+    run_all()
+    assert P.sasq_device_status() == 0
+    for got, ref in zip([pr[4] for pr in probs] + [yg], want):
+        assert torch.equal(got.view(torch.int16), ref.view(torch.int16))
