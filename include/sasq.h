@@ -241,6 +241,20 @@ SASQ_API int sasq_static_w8a8_linear_per_channel(const void* x, const int8_t* w,
                                                  int32_t* acc_out, int64_t T, int64_t N, int64_t K, int dt, int bits,
                                                  void* workspace, size_t ws_bytes, void* stream);
 
+/* Bytes of scratch sasq_fakequant_linear_fp_weights needs for this shape. */
+SASQ_API size_t sasq_fakequant_linear_fp_weights_workspace(int64_t T, int64_t N, int64_t K);
+
+/* The "FP weights" form of the quantized linear (Table 3; Eq. 5 and 6: quantization seen as a transform of the
+ * activations alone): the activations go through the fake-quant operator, the weights stay 16-bit floating point:
+ *   x'[t,k] = narrow( fl32(c(x[t,k]) * s) )                       (sasq_fakequant_fwd, bit for bit)
+ *   y[t,n]  = narrow( sum_k x'[t,k] * w[n,k] (+ bias[n]) )        products exact, fp32 accumulation on the tensor
+ *                                                                  cores (order unspecified), bias added in fp32
+ * x: [T, K], w: [N, K], bias: [N] or NULL, y: [T, N], all of `dt`; x_scale_dev: one fp32.  Constraints: K % 8 == 0,
+ * N % 8 == 0 (otherwise SASQ_ERR_UNSUPPORTED).  The workspace receives x'.  Two launches. */
+SASQ_API int sasq_fakequant_linear_fp_weights(const void* x, const void* w, const float* x_scale_dev, const void* bias,
+                                              void* y, int64_t T, int64_t N, int64_t K, int dt, int bits,
+                                              void* workspace, size_t ws_bytes, void* stream);
+
 /* Bytes of scratch sasq_static_w8a8_linear_grouped needs for this shape. */
 SASQ_API size_t sasq_static_w8a8_linear_grouped_workspace(int64_t T, int64_t N, int64_t K);
 

@@ -308,3 +308,20 @@ def w8a8_linear_per_channel(x: np.ndarray, tag: int, w_int: np.ndarray, w_scale:
     acc = int_gemm(codes.astype(np.int8), w_int)
     y, _ = dequant(acc, w_scale, 1.0, tag, bias)
     return y, acc
+
+
+def fp_weights_linear(x: np.ndarray, tag: int, w: np.ndarray, s: float, bits: int = 8, bias: np.ndarray | None = None):
+    """Table 3's "FP weights" form (Eq. 5 and 6: quantization as a transform of the activations alone):
+    Y = g(X) W^T with X' = g(X) the fake-quantized activations (the pinned forward) and the weights left in their
+    16-bit floating-point type.  The contraction is a library matmul in float64; returns the float64 result before
+    any narrowing, and sum_k |x'[t,k] w[n,k]| for error bounds."""
+    xq, _ = fakequant_fwd(x, tag, s, bits, want_codes=False)
+    a = widen(xq, tag).astype(np.float64)
+    b = widen(_u16(w), tag).astype(np.float64)
+    y = a @ b.T
+    mag = np.abs(a) @ np.abs(b).T
+    if bias is not None:
+        bv = widen(_u16(bias), tag).astype(np.float64)
+        y = y + bv[None, :]
+        mag = mag + np.abs(bv)[None, :]
+    return y, mag

@@ -24,7 +24,8 @@ __all__ = [
     "SASQ_WITHOUT_CLAMP", "sasq_dynamic_w8a8_linear_workspace", "sasq_dynamic_w8a8_linear", "sasq_debug_set_wait_limit", "PcDesc", "sasq_fakequant_per_channel_multi_workspace",
     "sasq_fakequant_fwd_bwd_per_channel_multi", "sasq_static_w8a8_linear_per_channel_workspace",
     "sasq_static_w8a8_linear_per_channel", "sasq_static_w8a8_linear_grouped_workspace",
-    "sasq_static_w8a8_linear_grouped", "LinearDesc", "sasq_static_w8a8_linear_multi_workspace",
+    "sasq_static_w8a8_linear_grouped", "sasq_fakequant_linear_fp_weights_workspace",
+    "sasq_fakequant_linear_fp_weights", "LinearDesc", "sasq_static_w8a8_linear_multi_workspace",
     "sasq_static_w8a8_linear_multi", "sasq_static_w8a8_linear_multi_launches", "sasq_set_gang_launch", "LinearProblems", "QuantTensors",
 ]
 
@@ -131,6 +132,10 @@ def load_library() -> ctypes.CDLL:
     L.sasq_fakequant_fwd_bwd_per_channel_multi.argtypes = [ctypes.POINTER(PcDesc), i32, i32, i32, i32, vp, sz, vp]
     L.sasq_debug_set_wait_limit.restype = ctypes.c_longlong
     L.sasq_debug_set_wait_limit.argtypes = [ctypes.c_longlong]
+    L.sasq_fakequant_linear_fp_weights_workspace.restype = sz
+    L.sasq_fakequant_linear_fp_weights_workspace.argtypes = [i64, i64, i64]
+    L.sasq_fakequant_linear_fp_weights.restype = i32
+    L.sasq_fakequant_linear_fp_weights.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, sz, vp]
     L.sasq_static_w8a8_linear_grouped_workspace.restype = sz
     L.sasq_static_w8a8_linear_grouped_workspace.argtypes = [i64, i64, i64]
     L.sasq_static_w8a8_linear_grouped.restype = i32
@@ -396,6 +401,28 @@ def sasq_static_w8a8_linear(x, w, w_scale, x_scale, y, bias=None, acc_out=None, 
     _check(load_library().sasq_static_w8a8_linear(_ptr(x), _ptr(w), _ptr(w_scale), _ptr(x_scale), _ptr(bias), _ptr(y),
                                                   _ptr(acc_out), T, N, K, _dt(x), int(bits), _ptr(workspace),
                                                   _nbytes(workspace), _stream(stream)), "sasq_static_w8a8_linear")
+
+
+def sasq_fakequant_linear_fp_weights_workspace(T: int, N: int, K: int) -> int:
+    return int(load_library().sasq_fakequant_linear_fp_weights_workspace(int(T), int(N), int(K)))
+
+
+def sasq_fakequant_linear_fp_weights(x, w, x_scale, y, bias=None, workspace=None, bits: int = 8, stream=None) -> None:
+    """Table 3's "FP weights" form: fake-quantized activations times 16-bit weights; x [T, K], w [N, K], y [T, N]."""
+    _dev(x, "x"); _dev(w, "w", x.dtype); _dev(x_scale, "x_scale", torch.float32); _dev(y, "y", x.dtype)
+    if bias is not None:
+        _dev(bias, "bias", x.dtype)
+    if workspace is not None:
+        _dev(workspace, "workspace")
+    if x.dim() != 2 or w.dim() != 2 or x.shape[1] != w.shape[1]:
+        raise ValueError("x must be [T, K] and w [N, K]")
+    T, K = x.shape
+    N = w.shape[0]
+    if tuple(y.shape) != (T, N) or (bias is not None and bias.numel() != N):
+        raise ValueError("y must be [T, N] and bias [N]")
+    _check(load_library().sasq_fakequant_linear_fp_weights(_ptr(x), _ptr(w), _ptr(x_scale), _ptr(bias), _ptr(y), T, N, K,
+                                                           _dt(x), int(bits), _ptr(workspace), _nbytes(workspace),
+                                                           _stream(stream)), "sasq_fakequant_linear_fp_weights")
 
 
 def sasq_static_w8a8_linear_grouped_workspace(T: int, N: int, K: int) -> int:

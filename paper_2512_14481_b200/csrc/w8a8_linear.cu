@@ -118,10 +118,14 @@ __device__ __forceinline__ bool epilogue_all_ok(bool ok) {
     return r != 0;
 }
 
-template <bool BF>
+// FPW = true: the "FP weights" form (Table 3, Eq. 5): both operands are 16-bit floating point (A = the fake-quantized
+// activations X' = g(X), B = the weights left as they are), kind::f16 MMAs with fp32 accumulators, no factors in the
+// epilogue.  A stage row is still 128 bytes: 64 elements, four MMAs of K = 16.
+template <bool BF, bool FPW>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 w8a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                  const __grid_constant__ LinearParams p) {
+    constexpr int KB_ELEMS = FPW ? BK / 2 : BK;          // elements of K per stage (the maps count in elements)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     SharedTail* tail = reinterpret_cast<SharedTail*>(tiles + (size_t)STAGES * STAGE_BYTES);
@@ -168,8 +172,8 @@ w8a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     uint8_t* a_dst = tiles + (size_t)stage * STAGE_BYTES;
                     uint8_t* b_dst = a_dst + A_STAGE_BYTES;
                     ptx::mbar_arrive_expect_tx(&tail->full[stage], STAGE_BYTES);
-                    ptx::tma_load_2d(a_dst, &tmap_a, &tail->full[stage], kb * BK, m_blk * BM);
-                    ptx::tma_load_2d(b_dst, &tmap_w, &tail->full[stage], kb * BK, n_blk * BN);
+                    ptx::tma_load_2d(a_dst, &tmap_a, &tail->full[stage], kb * KB_ELEMS, m_blk * BM);
+                    ptx::tma_load_2d(b_dst, &tmap_w, &tail->full[stage], kb * KB_ELEMS, n_blk * BN);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -190,7 +194,7 @@ w8a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (ptx::elect_one()) {
-            constexpr uint32_t idesc = ptx::idesc_i8(BM, BN);
+            constexpr uint32_t idesc = FPW ? ptx::idesc_f16(BM, BN, BF) : ptx::idesc_i8(BM, BN);
             const uint64_t a_desc0 = ptx::smem_desc_k_major_sw128(ptx::smem_u32(tiles));
             const uint64_t b_desc0 = ptx::smem_desc_k_major_sw128(ptx::smem_u32(tiles) + A_STAGE_BYTES);
             int stage = 0;
@@ -211,10 +215,18 @@ w8a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     ptx::tc_fence_after_sync();
                     const uint64_t a_desc = a_desc0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
                     const uint64_t b_desc = b_desc0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
-                    ptx::mma_i8_ss(d_tmem, a_desc, b_desc, idesc, accumulate);
-                    ptx::mma_i8_ss_acc(d_tmem, a_desc + 2, b_desc + 2, idesc);
-                    ptx::mma_i8_ss_acc(d_tmem, a_desc + 4, b_desc + 4, idesc);
-                    ptx::mma_i8_ss_acc(d_tmem, a_desc + 6, b_desc + 6, idesc);
+                    // either kind advances 32 bytes of K per MMA: +2 in the descriptor's address field
+                    if constexpr (FPW) {
+                        ptx::mma_f16_ss(d_tmem, a_desc, b_desc, idesc, accumulate);
+                        ptx::mma_f16_ss(d_tmem, a_desc + 2, b_desc + 2, idesc, 1u);
+                        ptx::mma_f16_ss(d_tmem, a_desc + 4, b_desc + 4, idesc, 1u);
+                        ptx::mma_f16_ss(d_tmem, a_desc + 6, b_desc + 6, idesc, 1u);
+                    } else {
+                        ptx::mma_i8_ss(d_tmem, a_desc, b_desc, idesc, accumulate);
+                        ptx::mma_i8_ss_acc(d_tmem, a_desc + 2, b_desc + 2, idesc);
+                        ptx::mma_i8_ss_acc(d_tmem, a_desc + 4, b_desc + 4, idesc);
+                        ptx::mma_i8_ss_acc(d_tmem, a_desc + 6, b_desc + 6, idesc);
+                    }
                     accumulate = 1u;
                     ptx::mma_commit(&tail->empty[stage]);          // stage reusable once these MMAs are done
                     if (kb == p.k_blocks - 1) ptx::mma_commit(&tail->tmem_full[buf]);
@@ -228,7 +240,7 @@ w8a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         const int quad = warp & 3;                      // TMEM lane quadrant this warp may read
         const int et = threadIdx.x - 64;                // 0..127
         const bool per_row = p.row_scale != nullptr;
-        const bool one_factor = !per_row && p.chan_inv == nullptr;       // one static factor for the whole tensor
+        const bool one_factor = !FPW && !per_row && p.chan_inv == nullptr;   // one static factor for the whole tensor
         const float sx = one_factor ? __ldg(p.x_scale) : 1.0f;
         if (one_factor && blockIdx.x == 0 && et == 0 && scale_is_bad(sx)) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
         bool ok = true;
@@ -242,7 +254,7 @@ w8a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             asm volatile("bar.sync 1, 128;" ::: "memory");
             for (int j = et; j < BN; j += EPI_THREADS) {
                 const int n = n0 + j;
-                tail->scale[j] = (n < p.N) ? __fmul_rn(sx, __ldg(p.w_scale + n)) : 0.0f;
+                if constexpr (!FPW) tail->scale[j] = (n < p.N) ? __fmul_rn(sx, __ldg(p.w_scale + n)) : 0.0f;
                 if (p.bias != nullptr)
                     tail->bias[j] = (n < p.N) ? widen1<BF>(__ldg(reinterpret_cast<const uint16_t*>(p.bias) + n)) : 0.0f;
             }
@@ -270,10 +282,16 @@ w8a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         uint32_t o[4];
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
-                            float f0 = __fmul_rn(__int2float_rn((int)v[j + 2 * q]),
-                                                 out_scale(per_row, s_row, tail->scale[c + j + 2 * q]));
-                            float f1 = __fmul_rn(__int2float_rn((int)v[j + 2 * q + 1]),
-                                                 out_scale(per_row, s_row, tail->scale[c + j + 2 * q + 1]));
+                            float f0, f1;
+                            if constexpr (FPW) {
+                                f0 = __uint_as_float(v[j + 2 * q]);
+                                f1 = __uint_as_float(v[j + 2 * q + 1]);
+                            } else {
+                                f0 = __fmul_rn(__int2float_rn((int)v[j + 2 * q]),
+                                               out_scale(per_row, s_row, tail->scale[c + j + 2 * q]));
+                                f1 = __fmul_rn(__int2float_rn((int)v[j + 2 * q + 1]),
+                                               out_scale(per_row, s_row, tail->scale[c + j + 2 * q + 1]));
+                            }
                             if (p.bias != nullptr) {
                                 f0 = __fadd_rn(f0, tail->bias[c + j + 2 * q]);
                                 f1 = __fadd_rn(f1, tail->bias[c + j + 2 * q + 1]);
@@ -1871,9 +1889,12 @@ bool single_kernel_ready(bool bf) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
     if (done[dev][bf]) return true;
-    const void* fn = bf ? reinterpret_cast<const void*>(w8a8_gemm_kernel<true>)
-                        : reinterpret_cast<const void*>(w8a8_gemm_kernel<false>);
-    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess)
+    const void* fn = bf ? reinterpret_cast<const void*>(w8a8_gemm_kernel<true, false>)
+                        : reinterpret_cast<const void*>(w8a8_gemm_kernel<false, false>);
+    const void* fn_fpw = bf ? reinterpret_cast<const void*>(w8a8_gemm_kernel<true, true>)
+                            : reinterpret_cast<const void*>(w8a8_gemm_kernel<false, true>);
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(fn_fpw, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess)
         return false;
     done[dev][bf] = true;
     return true;
@@ -2251,8 +2272,8 @@ int linear_impl(const void* x, const int8_t* w, const float* w_scale, const floa
         const long long tiles = (long long)p.m_blocks * p.n_blocks;
         const int grid = (int)(tiles < sm_count ? tiles : sm_count);
         if (!single_kernel_ready(dt == SASQ_BF16)) return SASQ_ERR_CUDA;
-        if (dt == SASQ_BF16) w8a8_gemm_kernel<true><<<grid, NUM_THREADS, kSmemBytes, st>>>(tmap_a, tmap_w, p);
-        else w8a8_gemm_kernel<false><<<grid, NUM_THREADS, kSmemBytes, st>>>(tmap_a, tmap_w, p);
+        if (dt == SASQ_BF16) w8a8_gemm_kernel<true, false><<<grid, NUM_THREADS, kSmemBytes, st>>>(tmap_a, tmap_w, p);
+        else w8a8_gemm_kernel<false, false><<<grid, NUM_THREADS, kSmemBytes, st>>>(tmap_a, tmap_w, p);
     }
     if (cudaGetLastError() != cudaSuccess) return SASQ_ERR_CUDA;
     return SASQ_OK;
@@ -2402,6 +2423,59 @@ int sasq_static_w8a8_linear_multi_launches(int count, const sasq_linear_desc_t* 
         return SASQ_OK;
     });
     return launches;
+}
+
+size_t sasq_fakequant_linear_fp_weights_workspace(int64_t T, int64_t N, int64_t K) {
+    (void)N;
+    if (T <= 0 || K <= 0) return 0;
+    return (size_t)(T * K) * 2 + 256;           // the fake-quantized activations X', 16-bit
+}
+
+int sasq_fakequant_linear_fp_weights(const void* x, const void* w, const float* x_scale_dev, const void* bias, void* y,
+                                     int64_t T, int64_t N, int64_t K, int dt, int bits, void* workspace,
+                                     size_t ws_bytes, void* stream) {
+    using namespace sasq;
+    if (T < 0 || N <= 0 || K <= 0) return SASQ_ERR_INVALID_ARG;
+    if (dt != SASQ_F16 && dt != SASQ_BF16) return SASQ_ERR_INVALID_ARG;
+    if (bits < 2 || bits > 8) return SASQ_ERR_INVALID_ARG;
+    if (w == nullptr || x_scale_dev == nullptr || (T > 0 && (x == nullptr || y == nullptr))) return SASQ_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(y) || (reinterpret_cast<uintptr_t>(x_scale_dev) & 3u) ||
+        (reinterpret_cast<uintptr_t>(bias) & 1u))
+        return SASQ_ERR_INVALID_ARG;
+    if (K % 8 != 0 || N % 8 != 0 || T > (1 << 24) || N > (1 << 24) || K > (1 << 24)) return SASQ_ERR_UNSUPPORTED;
+    if (T == 0) return SASQ_OK;
+    if (workspace == nullptr || !aligned16(workspace) || ws_bytes < sasq_fakequant_linear_fp_weights_workspace(T, N, K))
+        return SASQ_ERR_WORKSPACE;
+    const int sm_count = device_sm_count_if_sm100();
+    if (sm_count <= 0) return SASQ_ERR_UNSUPPORTED;
+    int* status = status_word_ptr();
+    if (status == nullptr) return SASQ_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool bf = dt == SASQ_BF16;
+    if (!single_kernel_ready(bf)) return SASQ_ERR_CUDA;
+
+    // 1. X' = g(X): the fake-quant forward (Eq. 1, Sec. 4.2) into the workspace; 2. Y = X' W^T on the tensor cores
+    void* xq = reinterpret_cast<void*>((reinterpret_cast<uintptr_t>(workspace) + 127) & ~uintptr_t(127));
+    const int rc = sasq_fakequant_fwd(x, xq, T * K, dt, x_scale_dev, bits, stream);
+    if (rc != SASQ_OK) return rc;
+    LinearParams p{};
+    p.bias = bias;
+    p.y = y;
+    p.T = (int)T; p.N = (int)N; p.K = (int)K;
+    p.k_blocks = (int)((K * 2 + BK - 1) / BK);
+    p.m_blocks = (int)((T + BM - 1) / BM);
+    p.n_blocks = (int)((N + BN - 1) / BN);
+    p.status = status;
+    p.wait_limit = g_wait_limit.load(std::memory_order_relaxed);
+    CUtensorMap tmap_a, tmap_w;
+    if (!make_tmap_generic(&tmap_a, xq, T, K, BM, BK / 2, 2) || !make_tmap_generic(&tmap_w, w, N, K, BN, BK / 2, 2))
+        return SASQ_ERR_CUDA;
+    const long long tiles = (long long)p.m_blocks * p.n_blocks;
+    const int grid = (int)(tiles < sm_count ? tiles : sm_count);
+    if (bf) w8a8_gemm_kernel<true, true><<<grid, NUM_THREADS, kSmemBytes, st>>>(tmap_a, tmap_w, p);
+    else w8a8_gemm_kernel<false, true><<<grid, NUM_THREADS, kSmemBytes, st>>>(tmap_a, tmap_w, p);
+    if (cudaGetLastError() != cudaSuccess) return SASQ_ERR_CUDA;
+    return SASQ_OK;
 }
 
 size_t sasq_static_w8a8_linear_grouped_workspace(int64_t T, int64_t N, int64_t K) {
