@@ -346,6 +346,20 @@ SASQ_API size_t sasq_absmax_scale_workspace(int64_t numel);
 SASQ_API int sasq_absmax_scale(const void* x, int64_t numel, int dt, int bits, float* scale_out_dev, void* workspace,
                                size_t ws_bytes, void* stream);
 
+/* The same per channel (column of x[T, K]), the granularity of the paper's experiments (Sec. 5.1):
+ * scales_out_dev[k] = max_t |x[t,k]| / Qp in fp32 (0 for an all-zero column or T == 0).  x: [T, K] of `dt`,
+ * K % 8 == 0; scales_out_dev: [K] fp32, also used as scratch while the call runs. */
+SASQ_API int sasq_absmax_scale_per_channel(const void* x, int64_t T, int64_t K, int dt, int bits,
+                                           float* scales_out_dev, void* stream);
+
+/* Running mean for the initialisation of Sec. 4.1 ("the average of the factors of the calibration batches"),
+ * kept on the device: fed the factors of batch number `count` (1, 2, ...) it turns the mean of the first
+ * count - 1 batches into the mean of the first count:
+ *   mean[i] = value[i]                                   if count == 1
+ *   mean[i] = mean[i] + (value[i] - mean[i]) / count     otherwise (fp32)
+ * mean_dev, value_dev: [n] fp32 (one entry per tensor, or per channel). */
+SASQ_API int sasq_running_mean(float* mean_dev, const float* value_dev, int n, int count, void* stream);
+
 /* Per-output-channel symmetric weight quantizer (Eq. 1 applied to each column of
  * the paper's K x N weight, i.e. each row of w[N, K]; weights are always
  * quantized per channel, Sec. 5.1):  w_scale[n] = max_k |w[n,k]| / Qp (1 for an

@@ -25,7 +25,7 @@ __all__ = [
     "sasq_fakequant_fwd_bwd_per_channel_multi", "sasq_static_w8a8_linear_per_channel_workspace",
     "sasq_static_w8a8_linear_per_channel", "sasq_static_w8a8_linear_grouped_workspace",
     "sasq_static_w8a8_linear_grouped", "sasq_fakequant_linear_fp_weights_workspace",
-    "sasq_fakequant_linear_fp_weights", "LinearDesc", "sasq_static_w8a8_linear_multi_workspace",
+    "sasq_fakequant_linear_fp_weights", "sasq_absmax_scale_per_channel", "sasq_running_mean", "LinearDesc", "sasq_static_w8a8_linear_multi_workspace",
     "sasq_static_w8a8_linear_multi", "sasq_static_w8a8_linear_multi_launches", "sasq_set_gang_launch", "LinearProblems", "QuantTensors",
 ]
 
@@ -604,6 +604,30 @@ def sasq_set_gang_launch(on: bool) -> bool:
 def sasq_device_status(stream=None) -> int:
     """Synchronises the stream; returns and clears the sticky device status (0 = OK)."""
     return int(load_library().sasq_device_status(_stream(stream)))
+
+
+def sasq_absmax_scale_per_channel(x, scales_out, bits: int = 8, stream=None) -> None:
+    """scales_out[k] = max_t |x[t, k]| / Qp (Eq. 1 per channel) of one calibration batch; x [T, K]."""
+    _dev(x, "x"); _dev(scales_out, "scales_out", torch.float32)
+    if x.dim() != 2 or scales_out.numel() != x.shape[1]:
+        raise ValueError("x must be [T, K] and scales_out [K]")
+    L = load_library()
+    L.sasq_absmax_scale_per_channel.restype = ctypes.c_int
+    L.sasq_absmax_scale_per_channel.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_int,
+                                                ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p]
+    _check(L.sasq_absmax_scale_per_channel(_ptr(x), x.shape[0], x.shape[1], _dt(x), int(bits), _ptr(scales_out),
+                                           _stream(stream)), "sasq_absmax_scale_per_channel")
+
+
+def sasq_running_mean(mean, value, count: int, stream=None) -> None:
+    """mean <- mean of the first `count` values, given the mean of the first count - 1 and the count-th value."""
+    _dev(mean, "mean", torch.float32); _dev(value, "value", torch.float32)
+    if mean.numel() != value.numel():
+        raise ValueError("mean and value must have the same number of elements")
+    L = load_library()
+    L.sasq_running_mean.restype = ctypes.c_int
+    L.sasq_running_mean.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_void_p]
+    _check(L.sasq_running_mean(_ptr(mean), _ptr(value), mean.numel(), int(count), _stream(stream)), "sasq_running_mean")
 
 
 def sasq_absmax_scale_workspace(numel: int) -> int:

@@ -56,6 +56,47 @@ __global__ void __launch_bounds__(kThreads) absmax_final_kernel(const float* __r
     if (threadIdx.x == 0) scale_out[0] = __fdiv_rn(m, qp);
 }
 
+// Max-based factor per channel (column of x[T, K]).  A thread owns 8 adjacent channels (one 128-bit word per row)
+// and walks down the rows of its block's row group; the groups meet in an atomic max on the bit patterns of the
+// (non-negative) maxima, whose integer order is their order as floats.
+template <bool BF>
+__global__ void __launch_bounds__(kThreads) absmax_channels_kernel(const uint4* __restrict__ x, int T, int vec_per_row,
+                                                                   int rows_per_group, unsigned* __restrict__ max_bits) {
+    const int cv = blockIdx.x * kThreads + threadIdx.x;          // which 8-channel word of a row
+    if (cv >= vec_per_row) return;
+    const int r0 = blockIdx.y * rows_per_group;
+    const int r1 = r0 + rows_per_group < T ? r0 + rows_per_group : T;
+    float m[8] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};
+    for (int r = r0; r < r1; ++r) {
+        const uint4 v = x[(size_t)r * vec_per_row + cv];
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float2 f = widen2<BF>(w[j]);
+            m[2 * j] = fmaxf(m[2 * j], fabsf(f.x));
+            m[2 * j + 1] = fmaxf(m[2 * j + 1], fabsf(f.y));
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) atomicMax(max_bits + 8 * cv + j, __float_as_uint(m[j]));
+}
+
+// bit patterns of the maxima -> factors, in place: s[k] = max / Qp
+__global__ void __launch_bounds__(kThreads) absmax_channels_final_kernel(unsigned* __restrict__ max_bits, int K, float qp) {
+    const int k = blockIdx.x * kThreads + threadIdx.x;
+    if (k < K) max_bits[k] = __float_as_uint(__fdiv_rn(__uint_as_float(max_bits[k]), qp));
+}
+
+// avg[i] <- avg[i] + (value[i] - avg[i]) / count: the mean of the first `count` values once each has been fed in turn
+__global__ void __launch_bounds__(kThreads) running_mean_kernel(float* __restrict__ avg, const float* __restrict__ value,
+                                                                int n, float count) {
+    const int i = blockIdx.x * kThreads + threadIdx.x;
+    if (i < n) {
+        const float a = avg[i];
+        avg[i] = count <= 1.0f ? value[i] : __fadd_rn(a, __fdiv_rn(__fsub_rn(value[i], a), count));
+    }
+}
+
 // one block per output channel (row of w[N, K])
 __global__ void __launch_bounds__(kThreads) quantize_weight_kernel(const float* __restrict__ w, int8_t* __restrict__ w_int,
                                                                    float* __restrict__ w_scale, long long K, float qn,
@@ -154,6 +195,56 @@ int sasq_absmax_scale(const void* x, int64_t numel, int dt, int bits, float* sca
         absmax_partial_kernel<false><<<(int)blocks, kThreads, 0, st>>>(static_cast<const uint16_t*>(x), numel, partial);
     if (cudaGetLastError() != cudaSuccess) return SASQ_ERR_CUDA;
     absmax_final_kernel<<<1, kThreads, 0, st>>>(partial, (int)blocks, (float)((1 << (bits - 1)) - 1), scale_out_dev);
+    if (cudaGetLastError() != cudaSuccess) return SASQ_ERR_CUDA;
+    return SASQ_OK;
+}
+
+int sasq_absmax_scale_per_channel(const void* x, int64_t T, int64_t K, int dt, int bits, float* scales_out_dev,
+                                  void* stream) {
+    using namespace sasq;
+    if (T < 0 || K <= 0 || scales_out_dev == nullptr || bits < 2 || bits > 8) return SASQ_ERR_INVALID_ARG;
+    if (dt != SASQ_F16 && dt != SASQ_BF16) return SASQ_ERR_INVALID_ARG;
+    if (T > 0 && (x == nullptr || !aligned16(x))) return SASQ_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(scales_out_dev) & 3u) return SASQ_ERR_INVALID_ARG;
+    if (K % 8 != 0 || T > (1 << 24) || K > (1 << 24)) return SASQ_ERR_UNSUPPORTED;
+    const int sm_count = device_sm_count_if_sm100();
+    if (sm_count <= 0) return SASQ_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned* bits_out = reinterpret_cast<unsigned*>(scales_out_dev);
+    if (cudaMemsetAsync(bits_out, 0, sizeof(unsigned) * (size_t)K, st) != cudaSuccess) return SASQ_ERR_CUDA;
+    if (T > 0) {
+        const int vec = (int)(K / 8);
+        const int col_blocks = (vec + kThreads - 1) / kThreads;
+        // enough row groups to fill the GPU a few times over, at least 16 rows each
+        long long groups = ((long long)sm_count * 8 + col_blocks - 1) / col_blocks;
+        if (groups > (T + 15) / 16) groups = (T + 15) / 16;
+        if (groups < 1) groups = 1;
+        if (groups > 65535) groups = 65535;
+        const int rows_per_group = (int)((T + groups - 1) / groups);
+        const dim3 grid((unsigned)col_blocks, (unsigned)((T + rows_per_group - 1) / rows_per_group), 1);
+        if (dt == SASQ_BF16)
+            absmax_channels_kernel<true><<<grid, kThreads, 0, st>>>(static_cast<const uint4*>(x), (int)T, vec,
+                                                                   rows_per_group, bits_out);
+        else
+            absmax_channels_kernel<false><<<grid, kThreads, 0, st>>>(static_cast<const uint4*>(x), (int)T, vec,
+                                                                    rows_per_group, bits_out);
+        if (cudaGetLastError() != cudaSuccess) return SASQ_ERR_CUDA;
+    }
+    absmax_channels_final_kernel<<<(unsigned)((K + kThreads - 1) / kThreads), kThreads, 0, st>>>(
+        bits_out, (int)K, (float)((1 << (bits - 1)) - 1));
+    if (cudaGetLastError() != cudaSuccess) return SASQ_ERR_CUDA;
+    return SASQ_OK;
+}
+
+int sasq_running_mean(float* mean_dev, const float* value_dev, int n, int count, void* stream) {
+    using namespace sasq;
+    if (n < 0 || count < 1 || (n > 0 && (mean_dev == nullptr || value_dev == nullptr))) return SASQ_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(mean_dev) & 3u) || (reinterpret_cast<uintptr_t>(value_dev) & 3u))
+        return SASQ_ERR_INVALID_ARG;
+    if (n == 0) return SASQ_OK;
+    if (device_sm_count_if_sm100() <= 0) return SASQ_ERR_UNSUPPORTED;
+    running_mean_kernel<<<(unsigned)((n + kThreads - 1) / kThreads), kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        mean_dev, value_dev, n, (float)count);
     if (cudaGetLastError() != cudaSuccess) return SASQ_ERR_CUDA;
     return SASQ_OK;
 }
