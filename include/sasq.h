@@ -282,8 +282,10 @@ SASQ_API size_t sasq_dynamic_w8a8_linear_workspace(int64_t T, int64_t N, int64_t
  *   X_int[t,k] = int8(c(x[t,k])) with s = s_t,   acc[t,n] = sum_k X_int[t,k] * w[n,k]
  *   y[t,n]     = narrow( fl32(acc) * fl32(s_t * w_scale[n]) (+ bias[n]) )
  * Arguments as for sasq_static_w8a8_linear, without x_scale_dev.  row_scale_out: [T] fp32 that receives the
- * factors, or NULL (they are then kept in the workspace).  One extra launch computes the factors and the codes (a
- * row's factor needs the whole row first). */
+ * factors, or NULL (they are then kept in the workspace).  For T <= 128 (the generation phase) everything runs in
+ * one launch: the rows are dealt to the CTAs of the GEMM kernel, whose quantizer warps find a row's factor and write
+ * its codes.  For larger T one extra launch computes the factors and the codes (a row's factor needs the whole row
+ * first). */
 SASQ_API int sasq_dynamic_w8a8_linear(const void* x, const int8_t* w, const float* w_scale, const void* bias, void* y,
                                       float* row_scale_out, int32_t* acc_out, int64_t T, int64_t N, int64_t K, int dt,
                                       int bits, void* workspace, size_t ws_bytes, void* stream);

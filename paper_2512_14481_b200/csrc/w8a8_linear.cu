@@ -1295,6 +1295,7 @@ struct DecodeTail {
     uint32_t tmem_base;
     volatile int abort_flag;
     int is_last_cta;
+    float row_max[4];    // dynamic per-token factors: the four quantizer warps' maxima of the row in hand
 };
 
 struct DecodeParams {
@@ -1311,7 +1312,11 @@ struct DecodeParams {
     unsigned* ready;     // [1] 16-element items quantized and visible; zero at launch
     unsigned* done;
     float qn, qp;
+    float* row_scale_out;   // non-NULL: dynamic per-token factors, computed here (a CTA's four quantizer warps per
+                            // row) and written there; lp.row_scale points at the same array for the epilogue
 };
+
+constexpr int D_DYN_WORDS = 12;   // 128-bit words of a row a quantizer thread keeps in registers between the two passes
 
 __device__ __forceinline__ bool wait_bounded_d(uint64_t* bar, uint32_t parity, DecodeTail* tail, const LinearParams& p) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
@@ -1463,7 +1468,64 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
         const bool one_factor = !per_row && p.chan_inv == nullptr;       // one static factor for the whole tensor
         const float sx = one_factor ? __ldg(p.x_scale) : 1.0f;
         if (one_factor && blockIdx.x == 0 && et == 0 && scale_is_bad(sx)) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
-        if (dp.x != nullptr) {
+        if (dp.x != nullptr && dp.row_scale_out != nullptr) {
+            // Dynamic per-token quantization (Sec. 4.4, generation phase) inside the launch: the rows are dealt to
+            // the CTAs, and the 128 quantizer threads of a CTA take a row together.  The row's factor is its own
+            // max-based one, s_t = max_k |x[t,k]| / Qp (Eq. 1; an all-zero row takes s_t = 1).  Each thread keeps its
+            // words of the row in registers between the maximum and the quantization (rows longer than
+            // 128 x D_DYN_WORDS words read the rest a second time).
+            const int vec = p.K >> 3;
+            unsigned rows_done = 0;
+            for (int r = blockIdx.x; r < p.T; r += gridDim.x) {
+                const uint4* row = reinterpret_cast<const uint4*>(dp.x) + (size_t)r * vec;
+                uint4 keep[D_DYN_WORDS];
+                float m = 0.0f;
+#pragma unroll
+                for (int u = 0; u < D_DYN_WORDS; ++u) {
+                    const int i = et + 128 * u;
+                    if (i < vec) {
+                        keep[u] = row[i];
+                        const uint32_t w4[4] = {keep[u].x, keep[u].y, keep[u].z, keep[u].w};
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const float2 f = widen2<BF>(w4[q]);
+                            m = fmaxf(m, fmaxf(fabsf(f.x), fabsf(f.y)));
+                        }
+                    }
+                }
+                for (int i = et + 128 * D_DYN_WORDS; i < vec; i += 128) {
+                    const uint4 v = row[i];
+                    const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float2 f = widen2<BF>(w4[q]);
+                        m = fmaxf(m, fmaxf(fabsf(f.x), fabsf(f.y)));
+                    }
+                }
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, off));
+                if (lane == 0) tail->row_max[warp - 2] = m;
+                asm volatile("bar.sync 3, 128;" ::: "memory");
+                m = fmaxf(fmaxf(tail->row_max[0], tail->row_max[1]), fmaxf(tail->row_max[2], tail->row_max[3]));
+                const float sc = m > 0.0f ? __fdiv_rn(m, dp.qp) : 1.0f;
+                const float inv = __fdiv_rn(1.0f, sc);
+                if (et == 0) dp.row_scale_out[r] = sc;
+                uint2* orow = reinterpret_cast<uint2*>(dp.a_int8) + (size_t)r * vec;
+#pragma unroll
+                for (int u = 0; u < D_DYN_WORDS; ++u) {
+                    const int i = et + 128 * u;
+                    if (i < vec) orow[i] = quantize8<BF, false>(keep[u], inv, dp.qn, dp.qp);
+                }
+                for (int i = et + 128 * D_DYN_WORDS; i < vec; i += 128)
+                    orow[i] = quantize8<BF, false>(row[i], inv, dp.qn, dp.qp);
+                ++rows_done;
+                asm volatile("bar.sync 3, 128;" ::: "memory");      // row_max is free for the next row
+            }
+            asm volatile("fence.proxy.async.global;" ::: "memory");
+            __threadfence();
+            asm volatile("bar.sync 3, 128;" ::: "memory");          // every thread's codes are out and fenced
+            if (et == 0 && rows_done != 0) atomicAdd(dp.ready, rows_done * (unsigned)(p.K >> 4));
+        } else if (dp.x != nullptr) {
             const float inv = __fdiv_rn(1.0f, sx);
             const uint4* src = reinterpret_cast<const uint4*>(dp.x);
             uint4* dst = reinterpret_cast<uint4*>(dp.a_int8);
@@ -1562,7 +1624,8 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
                 for (int j = 0; j < 4; ++j) {
                     const int t = t0 + j;
                     if (t < p.T) {
-                        const float sct = per_row ? __fmul_rn(__ldg(p.row_scale + t), ws) : sc;
+                        // a plain load: in the dynamic mode other CTAs wrote the factors during this launch
+                        const float sct = per_row ? __fmul_rn(p.row_scale[t], ws) : sc;
                         float f = __fmul_rn(__int2float_rn(acc[j]), sct);
                         if (has_bias) f = __fadd_rn(f, bv);
                         reinterpret_cast<uint16_t*>(p.y)[(size_t)t * p.N + n] = narrow1<BF>(f);
@@ -2142,13 +2205,21 @@ int linear_impl(const void* x, const int8_t* w, const float* w_scale, const floa
             return SASQ_ERR_CUDA;
         chan_inv = inv;
     }
+    // dynamic factors at small T: the small-T kernel computes them itself (a CTA's quantizer warps per row), so the
+    // generation phase is one launch per linear
+    const bool dynamic_inside = dynamic && split > 0;
+    float* dyn_scales = nullptr;
     if (dynamic) {
-        // per-token factors and codes by a launch of their own (the factor of a row needs the whole row first)
-        float* rs = row_scale_out;
-        if (rs == nullptr) {
+        dyn_scales = row_scale_out;
+        if (dyn_scales == nullptr) {
             const uintptr_t after = reinterpret_cast<uintptr_t>(a_int8) + (uintptr_t)((T * K + 255) / 256 * 256);
-            rs = reinterpret_cast<float*>(after);
+            dyn_scales = reinterpret_cast<float*>(after);
         }
+        row_scale = dyn_scales;
+    }
+    if (dynamic && !dynamic_inside) {
+        // per-token factors and codes by a launch of their own (the factor of a row needs the whole row first)
+        float* rs = dyn_scales;
         cudaLaunchConfig_t cfg{};
         cfg.gridDim = dim3((unsigned)T, 1, 1);
         cfg.blockDim = dim3(256, 1, 1);
@@ -2164,8 +2235,7 @@ int linear_impl(const void* x, const int8_t* w, const float* w_scale, const floa
             qe = cudaLaunchKernelEx(&cfg, quantize_rows_dynamic_kernel<false>, static_cast<const uint4*>(x),
                                     reinterpret_cast<uint2*>(a_int8), rs, (int)K, qn, qp);
         if (qe != cudaSuccess) return SASQ_ERR_CUDA;
-        row_scale = rs;
-    } else if (!in_kernel_quantizer) {
+    } else if (!dynamic && !in_kernel_quantizer) {
         const long long n8 = (T * K) / 8;     // K % 16 == 0
         long long blocks = (n8 + 255) / 256;
         if (blocks > (long long)sm_count * 8) blocks = (long long)sm_count * 8;
@@ -2214,9 +2284,10 @@ int linear_impl(const void* x, const int8_t* w, const float* w_scale, const floa
         dp.a_int8 = a_int8;
         dp.qn = qn;
         dp.qp = qp;
-        if (in_kernel_quantizer) {
+        if (in_kernel_quantizer || dynamic_inside) {
             dp.x = static_cast<const uint16_t*>(x);
             if (!next_ready_slot(&dp.ready, &dp.done)) return SASQ_ERR_CUDA;
+            if (dynamic_inside) dp.row_scale_out = dyn_scales;
         }
         if (!make_tmap(&tmap_w, w, N, K, 128) || !make_tmap(&tmap_a, a_int8, T, K, dp.tp)) return SASQ_ERR_CUDA;
         cudaLaunchConfig_t cfg{};
