@@ -315,8 +315,10 @@ SASQ_API size_t sasq_static_w8a8_linear_multi_workspace(int count, const sasq_li
  * of a problem and the drain of its last tiles overlap with the MMAs of its neighbours instead of idling the tensor
  * cores at every launch boundary.  A run that contains problems with T <= 128 shares a launch only if it has at
  * least two problems whose output tiles fill every resident CTA pair (the weights then stream through one launch
- * instead of one latency chain per linear); otherwise its problems are launched one by one, in order.  No problem
- * may read another's output.  descs_host: HOST memory, read before the call returns.  All problems share dt and bits.
+ * instead of one latency chain per linear); otherwise consecutive problems with the same T <= 128 whose 128-channel
+ * output tiles all fit the device at once (one CTA each; e.g. the q/k/v projections of a decode step) share one
+ * launch of the small-T kernel, and what is left is launched one by one, in order.  No problem may read another's
+ * output.  descs_host: HOST memory, read before the call returns.  All problems share dt and bits.
  * Returns SASQ_ERR_INVALID_ARG / UNSUPPORTED / WORKSPACE as sasq_static_w8a8_linear does, checked for every problem
  * before anything is launched. */
 SASQ_API int sasq_static_w8a8_linear_multi(int count, const sasq_linear_desc_t* descs_host, int dt, int bits,

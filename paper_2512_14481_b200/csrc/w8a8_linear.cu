@@ -1298,18 +1298,30 @@ struct DecodeTail {
     float row_max[4];    // dynamic per-token factors: the four quantizer warps' maxima of the row in hand
 };
 
-struct DecodeParams {
+// One launch may carry several independent problems with the same T (the q/k/v projections of a decode step, say):
+// the 128-channel tiles of all of them form one list of clusters, and every CTA helps to quantize every problem's x.
+constexpr int kMaxDecodeGroup = 8;
+struct DecodeProblem {
     LinearParams lp;
+    const uint16_t* x;   // NULL: the codes in a_int8 were written by an earlier launch
+    uint8_t* a_int8;
+    int tile_begin;      // 128-channel tiles of the problems before this one
+};
+struct DecodeMaps {
+    CUtensorMap w[kMaxDecodeGroup], x[kMaxDecodeGroup];
+};
+struct DecodeParams {
+    int count;
+    DecodeProblem prob[kMaxDecodeGroup];
     int tp;              // T rounded up to a multiple of 16: N of the MMA
     int stages;
     int split;           // CTAs per cluster = K slices
-    int n_tiles;         // 128-channel tiles
+    int n_tiles;         // 128-channel tiles of all problems
     uint32_t tmem_cols;  // power of two >= max(32, tp)
     int slots_offset;    // byte offset of the reduction slots in the CTA's shared memory: behind the stages, never
                          // under them, because peers write there while this CTA may still be in its mainloop
-    const uint16_t* x;
-    uint8_t* a_int8;
-    unsigned* ready;     // [1] 16-element items quantized and visible; zero at launch
+    bool quantize;       // the activation quantizer runs inside this launch
+    unsigned* ready;     // [count] per problem: 16-element items quantized and visible; zero at launch
     unsigned* done;
     float qn, qp;
     float* row_scale_out;   // non-NULL: dynamic per-token factors, computed here (a CTA's four quantizer warps per
@@ -1337,12 +1349,18 @@ __device__ __forceinline__ bool wait_bounded_d(uint64_t* bar, uint32_t parity, D
 
 template <bool BF>
 __global__ void __launch_bounds__(D_THREADS, 1)
-w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
-                   const __grid_constant__ DecodeParams dp) {
+w8a8_decode_kernel(const __grid_constant__ DecodeMaps maps, const __grid_constant__ DecodeParams dp) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* ring = smem_raw;
     DecodeTail* tail = reinterpret_cast<DecodeTail*>(ring + D_RING_BYTES);
-    const LinearParams& p = dp.lp;
+    // the problem this cluster's tile belongs to
+    const int tile_all = blockIdx.x / dp.split;
+    int q_mine = 0;
+    while (q_mine + 1 < dp.count && tile_all >= dp.prob[q_mine + 1].tile_begin) ++q_mine;
+    const DecodeProblem& me = dp.prob[q_mine];
+    const LinearParams& p = me.lp;
+    const CUtensorMap* tmap_w = &maps.w[q_mine];
+    const CUtensorMap* tmap_x = &maps.x[q_mine];
     if ((ptx::smem_u32(ring) & 1023u) != 0) {       // uniform over the grid: every CTA returns before any barrier
         if (threadIdx.x == 0) atomicMax(p.status, (int)SASQ_ERR_CUDA);
         return;
@@ -1352,7 +1370,7 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int rank = (int)ptx::cluster_ctarank();
-    const int n_tile = blockIdx.x / dp.split;
+    const int n_tile = tile_all - me.tile_begin;
     const int n0 = n_tile * 128;
     const int stage_bytes = D_W_BYTES + dp.tp * BK;
     // this CTA's slice of the k-blocks
@@ -1367,8 +1385,8 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
         ptx::mbar_init(&tail->acc_full, 1);
         tail->abort_flag = 0;
         ptx::mbar_init_fence();
-        ptx::prefetch_tensormap(&tmap_w);
-        ptx::prefetch_tensormap(&tmap_x);
+        ptx::prefetch_tensormap(tmap_w);
+        ptx::prefetch_tensormap(tmap_x);
     }
     if (warp == 1) {
         ptx::tmem_alloc(&tail->tmem_base, dp.tmem_cols);
@@ -1381,7 +1399,7 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
     pdl_wait();                         // set-up done; from here on global memory of earlier kernels is used
 
     // 16-element items the in-kernel quantizer has to publish (none if the activations came quantized)
-    const unsigned items_total = dp.x != nullptr ? (unsigned)(((long long)p.T * p.K) >> 4) : 0u;
+    const unsigned items_total = dp.quantize ? (unsigned)(((long long)p.T * p.K) >> 4) : 0u;   // of this CTA's problem
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
@@ -1394,14 +1412,14 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
             int early = kb_end - kb_begin < dp.stages ? kb_end - kb_begin : dp.stages;
             for (int i = 0; i < early; ++i) {
                 ptx::mbar_arrive_expect_tx(&tail->full[i], (uint32_t)stage_bytes);
-                ptx::tma_load_2d(ring + (size_t)i * stage_bytes, &tmap_w, &tail->full[i], (kb_begin + i) * BK, n0);
+                ptx::tma_load_2d(ring + (size_t)i * stage_bytes, tmap_w, &tail->full[i], (kb_begin + i) * BK, n0);
             }
             if (items_total != 0) {
                 const long long t0 = clock64();
                 int polls = 0;
                 for (;;) {
                     unsigned v;
-                    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(dp.ready) : "memory");
+                    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(dp.ready + q_mine) : "memory");
                     if (v >= items_total) break;
                     if (p.wait_limit <= 0 || (++polls & 15) == 0) {
                         if (tail->abort_flag) { ok = false; break; }
@@ -1422,9 +1440,9 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
                     ok = wait_bounded_d(&tail->empty[stage], phase ^ 1u, tail, p);
                     if (!ok) break;
                     ptx::mbar_arrive_expect_tx(&tail->full[stage], (uint32_t)stage_bytes);
-                    ptx::tma_load_2d(w_dst, &tmap_w, &tail->full[stage], kb * BK, n0);
+                    ptx::tma_load_2d(w_dst, tmap_w, &tail->full[stage], kb * BK, n0);
                 }
-                ptx::tma_load_2d(w_dst + D_W_BYTES, &tmap_x, &tail->full[stage], kb * BK, 0);
+                ptx::tma_load_2d(w_dst + D_W_BYTES, tmap_x, &tail->full[stage], kb * BK, 0);
                 if (++stage == dp.stages) { stage = 0; phase ^= 1u; }
             }
             if (!ok) {      // copies in flight must land before the CTA's shared memory goes away
@@ -1464,11 +1482,7 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
     } else {
         // ---------------- activation quantizer, then epilogue (warps 2..5) ----------------
         const int et = threadIdx.x - 64;                       // 0..127
-        const bool per_row = p.row_scale != nullptr;
-        const bool one_factor = !per_row && p.chan_inv == nullptr;       // one static factor for the whole tensor
-        const float sx = one_factor ? __ldg(p.x_scale) : 1.0f;
-        if (one_factor && blockIdx.x == 0 && et == 0 && scale_is_bad(sx)) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
-        if (dp.x != nullptr && dp.row_scale_out != nullptr) {
+        if (dp.quantize && dp.row_scale_out != nullptr) {
             // Dynamic per-token quantization (Sec. 4.4, generation phase) inside the launch: the rows are dealt to
             // the CTAs, and the 128 quantizer threads of a CTA take a row together.  The row's factor is its own
             // max-based one, s_t = max_k |x[t,k]| / Qp (Eq. 1; an all-zero row takes s_t = 1).  Each thread keeps its
@@ -1477,7 +1491,7 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
             const int vec = p.K >> 3;
             unsigned rows_done = 0;
             for (int r = blockIdx.x; r < p.T; r += gridDim.x) {
-                const uint4* row = reinterpret_cast<const uint4*>(dp.x) + (size_t)r * vec;
+                const uint4* row = reinterpret_cast<const uint4*>(me.x) + (size_t)r * vec;
                 uint4 keep[D_DYN_WORDS];
                 float m = 0.0f;
 #pragma unroll
@@ -1510,7 +1524,7 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
                 const float sc = m > 0.0f ? __fdiv_rn(m, dp.qp) : 1.0f;
                 const float inv = __fdiv_rn(1.0f, sc);
                 if (et == 0) dp.row_scale_out[r] = sc;
-                uint2* orow = reinterpret_cast<uint2*>(dp.a_int8) + (size_t)r * vec;
+                uint2* orow = reinterpret_cast<uint2*>(me.a_int8) + (size_t)r * vec;
 #pragma unroll
                 for (int u = 0; u < D_DYN_WORDS; ++u) {
                     const int i = et + 128 * u;
@@ -1524,31 +1538,43 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
             asm volatile("fence.proxy.async.global;" ::: "memory");
             __threadfence();
             asm volatile("bar.sync 3, 128;" ::: "memory");          // every thread's codes are out and fenced
-            if (et == 0 && rows_done != 0) atomicAdd(dp.ready, rows_done * (unsigned)(p.K >> 4));
-        } else if (dp.x != nullptr) {
-            const float inv = __fdiv_rn(1.0f, sx);
-            const uint4* src = reinterpret_cast<const uint4*>(dp.x);
-            uint4* dst = reinterpret_cast<uint4*>(dp.a_int8);
-            unsigned mine = 0;
-            for (unsigned i = blockIdx.x * 128u + (unsigned)et; i < items_total; i += gridDim.x * 128u) {
-                const uint4 a = ld_stream16(src + 2 * (size_t)i), b = ld_stream16(src + 2 * (size_t)i + 1);
-                uint2 lo, hi;
-                if (p.chan_inv != nullptr) {
-                    const float* ci = p.chan_inv + 16 * (i % (unsigned)(p.K >> 4));
-                    lo = quantize8_channels<BF>(a, ci, dp.qn, dp.qp);
-                    hi = quantize8_channels<BF>(b, ci + 8, dp.qn, dp.qp);
-                } else {
-                    lo = quantize8<BF, false>(a, inv, dp.qn, dp.qp);
-                    hi = quantize8<BF, false>(b, inv, dp.qn, dp.qp);
+            if (et == 0 && rows_done != 0) atomicAdd(dp.ready + q_mine, rows_done * (unsigned)(p.K >> 4));
+        } else if (dp.quantize) {
+            // every CTA takes its share of every problem's x, in problem order
+            for (int q = 0; q < dp.count; ++q) {
+                const DecodeProblem& pr = dp.prob[q];
+                const LinearParams& lp = pr.lp;
+                const bool one = lp.chan_inv == nullptr;                 // one static factor for the whole tensor
+                const float sxq = one ? __ldg(lp.x_scale) : 1.0f;
+                if (one && blockIdx.x == 0 && et == 0 && scale_is_bad(sxq)) atomicMax(lp.status, (int)SASQ_ERR_BAD_SCALE);
+                const float inv = __fdiv_rn(1.0f, sxq);
+                const uint4* src = reinterpret_cast<const uint4*>(pr.x);
+                uint4* dst = reinterpret_cast<uint4*>(pr.a_int8);
+                const unsigned items = (unsigned)(((long long)lp.T * lp.K) >> 4);
+                unsigned mine = 0;
+                for (unsigned i = blockIdx.x * 128u + (unsigned)et; i < items; i += gridDim.x * 128u) {
+                    const uint4 a = ld_stream16(src + 2 * (size_t)i), b = ld_stream16(src + 2 * (size_t)i + 1);
+                    uint2 lo, hi;
+                    if (lp.chan_inv != nullptr) {
+                        const float* ci = lp.chan_inv + 16 * (i % (unsigned)(lp.K >> 4));
+                        lo = quantize8_channels<BF>(a, ci, dp.qn, dp.qp);
+                        hi = quantize8_channels<BF>(b, ci + 8, dp.qn, dp.qp);
+                    } else {
+                        lo = quantize8<BF, false>(a, inv, dp.qn, dp.qp);
+                        hi = quantize8<BF, false>(b, inv, dp.qn, dp.qp);
+                    }
+                    dst[i] = make_uint4(lo.x, lo.y, hi.x, hi.y);
+                    ++mine;
                 }
-                dst[i] = make_uint4(lo.x, lo.y, hi.x, hi.y);
-                ++mine;
+                asm volatile("fence.proxy.async.global;" ::: "memory");
+                __threadfence();
+                // one add per warp
+                for (int off = 16; off > 0; off >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, off);
+                if (lane == 0 && mine != 0) atomicAdd(dp.ready + q, mine);
             }
-            asm volatile("fence.proxy.async.global;" ::: "memory");
-            __threadfence();
-            // one add per warp
-            for (int off = 16; off > 0; off >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, off);
-            if (lane == 0 && mine != 0) atomicAdd(dp.ready, mine);
+        } else if (blockIdx.x == 0 && et == 0 && p.row_scale == nullptr && p.chan_inv == nullptr &&
+                   scale_is_bad(__ldg(p.x_scale))) {
+            atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);             // codes from an earlier launch: check the factor
         }
 
         // epilogue part 1: this CTA's partial accumulators go from TMEM straight into the shared memory of the CTA
@@ -1644,9 +1670,9 @@ w8a8_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
         ptx::tmem_dealloc(tmem_base, dp.tmem_cols);
     }
     // the CTA that finishes last leaves the counters at zero for the next launch that draws them
-    if (dp.x != nullptr && threadIdx.x == 0) {
+    if (dp.quantize && threadIdx.x == 0) {
         if (atomicAdd(dp.done, 1u) == gridDim.x - 1) {
-            *dp.ready = 0u;
+            for (int q = 0; q < dp.count; ++q) dp.ready[q] = 0u;
             *dp.done = 0u;
         }
     }
@@ -2117,6 +2143,44 @@ int launch_pair_group(const GroupMaps& maps, const GroupParams& gp, int pairs, b
     return e == cudaSuccess ? SASQ_OK : SASQ_ERR_CUDA;
 }
 
+// One launch of the small-T kernel over the problems of `dp` (all with T rows; prob[].lp, x, a_int8, tile_begin,
+// n_tiles, quantize, qn, qp, row_scale_out and maps.w filled in by the caller): sets the shared geometry, draws the
+// counters, encodes the activation maps and launches n_tiles clusters of `split` CTAs.
+int launch_decode_group(DecodeMaps& maps, DecodeParams& dp, int T, int split, bool bf, cudaStream_t st) {
+    constexpr size_t kDecodeSmem = (size_t)D_RING_BYTES + sizeof(DecodeTail);
+    dp.tp = (T + 15) / 16 * 16;
+    const int stage_bytes = D_W_BYTES + dp.tp * BK;
+    const int slot_bytes = (128 * (dp.tp + 4) * 4 + 1023) & ~1023;          // S x (128 / S) rows of tp + 4 words
+    const int ring_bytes = D_RING_BYTES - slot_bytes;
+    dp.slots_offset = ring_bytes;
+    dp.stages = ring_bytes / stage_bytes < D_MAX_STAGES ? ring_bytes / stage_bytes : D_MAX_STAGES;
+    dp.split = split;
+    dp.tmem_cols = 32;
+    while ((int)dp.tmem_cols < dp.tp) dp.tmem_cols <<= 1;
+    if (dp.quantize && !next_ready_slot(&dp.ready, &dp.done)) return SASQ_ERR_CUDA;
+    for (int q = 0; q < dp.count; ++q)
+        if (!make_tmap(&maps.x[q], dp.prob[q].a_int8, T, dp.prob[q].lp.K, dp.tp)) return SASQ_ERR_CUDA;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)(dp.n_tiles * split), 1, 1);
+    cfg.blockDim = dim3(D_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = kDecodeSmem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[3];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)split;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1] = pdl_attribute();
+    attr[2].id = cudaLaunchAttributeCooperative;
+    attr[2].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = (dp.quantize && g_gang_launch.load(std::memory_order_relaxed)) ? 3 : 2;
+    cudaError_t e;
+    if (bf) e = cudaLaunchKernelEx(&cfg, w8a8_decode_kernel<true>, maps, dp);
+    else e = cudaLaunchKernelEx(&cfg, w8a8_decode_kernel<false>, maps, dp);
+    return e == cudaSuccess ? SASQ_OK : SASQ_ERR_CUDA;
+}
+
 // Cuts a list of problems into runs that fit one launch of the CTA-pair kernel (up to kMaxGroup problems,
 // kMaxRowBlocks row blocks, kGroupCodeBytes of int8 codes) and tells `visit(first, last, grouped)` for each run
 // whether it goes to that kernel in one launch: yes if all its problems have T > 128, or if it has small-T problems
@@ -2156,6 +2220,43 @@ int for_each_run(int count, const sasq_linear_desc_t* descs, int pairs, Visit vi
         }
         if (rc != SASQ_OK) return rc;
         first = last;
+    }
+    return SASQ_OK;
+}
+
+// Within a run that does not go to the CTA-pair kernel: consecutive problems with the same T <= 128 whose
+// 128-channel tiles all fit the device at once (one CTA each) share a launch of the small-T kernel, two to
+// kMaxDecodeGroup of them; `visit(first, last, together)` is told for each segment.  Everything else goes alone.
+template <typename Visit>
+int for_each_small_segment(int first, int last, const sasq_linear_desc_t* descs, int sm_count, Visit visit) {
+    int i = first;
+    while (i < last) {
+        const sasq_linear_desc_t& d = descs[i];
+        if (d.T == 0) { ++i; continue; }
+        int j = i + 1;
+        if (d.T <= BM) {
+            long long tiles = (d.N + 127) / 128;
+            int live = 1;
+            while (j < last && live < kMaxDecodeGroup) {
+                const sasq_linear_desc_t& e = descs[j];
+                if (e.T != 0) {
+                    if (e.T != d.T || tiles + (e.N + 127) / 128 > sm_count) break;
+                    tiles += (e.N + 127) / 128;
+                    ++live;
+                }
+                ++j;
+            }
+            if (live >= 2 && tiles <= sm_count) {
+                const int rc = visit(i, j, true);
+                if (rc != SASQ_OK) return rc;
+                i = j;
+                continue;
+            }
+            j = i + 1;
+        }
+        const int rc = visit(i, j, false);
+        if (rc != SASQ_OK) return rc;
+        i = j;
     }
     return SASQ_OK;
 }
@@ -2268,46 +2369,24 @@ int linear_impl(const void* x, const int8_t* w, const float* w_scale, const floa
     if (split > 0) {
         // small T: 128-channel tiles, K split over a cluster, activations quantized inside the kernel
         DecodeParams dp{};
+        DecodeMaps dmaps{};
         p.m_blocks = 1;
         p.n_blocks = n_tiles128;
-        dp.lp = p;
-        dp.tp = (int)((T + 15) / 16) * 16;
-        const int stage_bytes = D_W_BYTES + dp.tp * BK;
-        const int slot_bytes = (128 * (dp.tp + 4) * 4 + 1023) & ~1023;          // S x (128 / S) rows of tp + 4 words
-        const int ring_bytes = D_RING_BYTES - slot_bytes;
-        dp.slots_offset = ring_bytes;
-        dp.stages = ring_bytes / stage_bytes < D_MAX_STAGES ? ring_bytes / stage_bytes : D_MAX_STAGES;
-        dp.split = split;
+        dp.count = 1;
+        dp.prob[0].lp = p;
+        dp.prob[0].a_int8 = a_int8;
+        dp.prob[0].tile_begin = 0;
         dp.n_tiles = n_tiles128;
-        dp.tmem_cols = 32;
-        while ((int)dp.tmem_cols < dp.tp) dp.tmem_cols <<= 1;
-        dp.a_int8 = a_int8;
         dp.qn = qn;
         dp.qp = qp;
         if (in_kernel_quantizer || dynamic_inside) {
-            dp.x = static_cast<const uint16_t*>(x);
-            if (!next_ready_slot(&dp.ready, &dp.done)) return SASQ_ERR_CUDA;
+            dp.prob[0].x = static_cast<const uint16_t*>(x);
+            dp.quantize = true;
             if (dynamic_inside) dp.row_scale_out = dyn_scales;
         }
-        if (!make_tmap(&tmap_w, w, N, K, 128) || !make_tmap(&tmap_a, a_int8, T, K, dp.tp)) return SASQ_ERR_CUDA;
-        cudaLaunchConfig_t cfg{};
-        cfg.gridDim = dim3((unsigned)(n_tiles128 * split), 1, 1);
-        cfg.blockDim = dim3(D_THREADS, 1, 1);
-        cfg.dynamicSmemBytes = kDecodeSmem;
-        cfg.stream = st;
-        cudaLaunchAttribute attr[3];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = (unsigned)split;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        attr[1] = pdl_attribute();
-        attr[2].id = cudaLaunchAttributeCooperative;
-        attr[2].val.cooperative = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = (dp.x != nullptr && g_gang_launch.load(std::memory_order_relaxed)) ? 3 : 2;
-        if (dt == SASQ_BF16) e = cudaLaunchKernelEx(&cfg, w8a8_decode_kernel<true>, tmap_w, tmap_a, dp);
-        else e = cudaLaunchKernelEx(&cfg, w8a8_decode_kernel<false>, tmap_w, tmap_a, dp);
-        if (e != cudaSuccess) return SASQ_ERR_CUDA;
+        if (!make_tmap(&dmaps.w[0], w, N, K, 128)) return SASQ_ERR_CUDA;
+        const int rc = launch_decode_group(dmaps, dp, (int)T, split, dt == SASQ_BF16, st);
+        if (rc != SASQ_OK) return rc;
     } else if (T > BM) {
         // CTA pairs, 256-row blocks cut into evenly wide column tiles that fill whole waves of the resident pairs
         const int pairs = pair_capacity(dt == SASQ_BF16, sm_count);
@@ -2463,11 +2542,59 @@ int sasq_static_w8a8_linear_multi(int count, const sasq_linear_desc_t* descs_hos
         return launch_pair_group(maps, gp, pairs, bf, st, small_layout);
     };
 
+    // one launch of the small-T kernel for problems [first, last), all with the same T <= 128
+    auto run_small_group = [&](int first, int last) -> int {
+        DecodeParams dp{};
+        DecodeMaps dmaps{};
+        int T = 0, min_kblocks = 1 << 30;
+        for (int i = first; i < last; ++i) {
+            const sasq_linear_desc_t& d = descs_host[i];
+            if (d.T == 0) continue;
+            const int q = dp.count;
+            DecodeProblem& pr = dp.prob[q];
+            LinearParams& p = pr.lp;
+            p.w_scale = d.w_scale;
+            p.x_scale = d.x_scale;
+            p.bias = d.bias;
+            p.y = d.y;
+            p.T = (int)d.T; p.N = (int)d.N; p.K = (int)d.K;
+            p.k_blocks = (int)((d.K + BK - 1) / BK);
+            p.m_blocks = 1;
+            p.n_blocks = (int)((d.N + 127) / 128);
+            p.status = status;
+            p.wait_limit = wait_limit;
+            pr.x = static_cast<const uint16_t*>(d.x);
+            pr.a_int8 = reinterpret_cast<uint8_t*>(slice(i));
+            pr.tile_begin = dp.n_tiles;
+            if (!make_tmap(&dmaps.w[q], d.w, d.N, d.K, 128)) return SASQ_ERR_CUDA;
+            dp.n_tiles += p.n_blocks;
+            if (p.k_blocks < min_kblocks) min_kblocks = p.k_blocks;
+            T = (int)d.T;
+            dp.count = q + 1;
+        }
+        dp.quantize = true;
+        dp.qn = qn;
+        dp.qp = qp;
+        constexpr size_t kDecodeSmem = (size_t)D_RING_BYTES + sizeof(DecodeTail);
+        const int split = decode_split(bf, dp.n_tiles, min_kblocks, sm_count, kDecodeSmem);
+        if (split <= 0) {                        // cannot all be resident after all: one by one
+            int rc = SASQ_OK;
+            for (int i = first; i < last && rc == SASQ_OK; ++i)
+                if (descs_host[i].T > 0) rc = run_alone(i);
+            return rc;
+        }
+        return launch_decode_group(dmaps, dp, T, split, bf, st);
+    };
+
     return for_each_run(count, descs_host, pairs, [&](int first, int last, bool grouped) -> int {
         if (grouped) return run_group(first, last);
-        int rc = SASQ_OK;
-        for (int i = first; i < last && rc == SASQ_OK; ++i) rc = run_alone(i);
-        return rc;
+        return for_each_small_segment(first, last, descs_host, sm_count, [&](int a, int b, bool together) -> int {
+            if (together) return run_small_group(a, b);
+            int rc = SASQ_OK;
+            for (int i = a; i < b && rc == SASQ_OK; ++i)
+                if (descs_host[i].T > 0) rc = run_alone(i);
+            return rc;
+        });
     });
 }
 
@@ -2483,15 +2610,22 @@ int sasq_static_w8a8_linear_multi_launches(int count, const sasq_linear_desc_t* 
                 if (descs_host[i].T > 0) { ++launches; break; }
             return SASQ_OK;
         }
-        for (int i = first; i < last; ++i) {
-            const sasq_linear_desc_t& d = descs_host[i];
-            if (d.T == 0) continue;
-            // the activation quantizer runs inside the GEMM launch unless the row blocks (T > 128) or the
-            // 128-channel tiles (T <= 128) outnumber what its counters / the resident CTAs can hold
-            const bool inside = d.T > BM ? (d.T + PBM - 1) / PBM <= kMaxRowBlocks : (d.N + 127) / 128 <= 2 * num_pairs;
-            launches += inside ? 1 : 2;
-        }
-        return SASQ_OK;
+        return for_each_small_segment(first, last, descs_host, 2 * num_pairs, [&](int a, int b, bool together) -> int {
+            if (together) {
+                ++launches;
+                return SASQ_OK;
+            }
+            for (int i = a; i < b; ++i) {
+                const sasq_linear_desc_t& d = descs_host[i];
+                if (d.T == 0) continue;
+                // the activation quantizer runs inside the GEMM launch unless the row blocks (T > 128) or the
+                // 128-channel tiles (T <= 128) outnumber what its counters / the resident CTAs can hold
+                const bool inside =
+                    d.T > BM ? (d.T + PBM - 1) / PBM <= kMaxRowBlocks : (d.N + 127) / 128 <= 2 * num_pairs;
+                launches += inside ? 1 : 2;
+            }
+            return SASQ_OK;
+        });
     });
     return launches;
 }

@@ -118,6 +118,25 @@ def test_single_row_block_problems_take_the_cost_dealt_tile_lists():
     check_against_oracle(problems, tag)
 
 
+@pytest.mark.parametrize("tag", [oracle.F16, oracle.BF16])
+@pytest.mark.parametrize("T", [1, 16, 100])
+def test_same_t_small_problems_share_a_launch_of_the_small_t_kernel(tag, T):
+    """Too few tiles for the CTA pairs, but all 128-channel tiles fit the device: one launch of the small-T kernel
+    over three problems with different N and K (the K split is limited by the shortest), one with a bias."""
+    problems = [make_problem(T, 1032, 512, tag, 9900 + T),
+                make_problem(T, 520, 2048, tag, 9910 + T, with_bias=True),
+                make_problem(T, 2048, 256, tag, 9920 + T)]
+    assert P.sasq_static_w8a8_linear_multi_launches([(pr["T"], pr["N"], pr["K"]) for pr in problems]) == 1
+    check_against_oracle(problems, tag)
+
+
+def test_llama7b_qkv_at_decode_size_share_a_small_t_launch():
+    tag, T = oracle.BF16, 16
+    problems = [make_problem(T, 4096, 4096, tag, 9950 + i) for i in range(3)]
+    assert P.sasq_static_w8a8_linear_multi_launches([(pr["T"], pr["N"], pr["K"]) for pr in problems]) == 1
+    check_against_oracle(problems, tag)
+
+
 def test_llama7b_layer_at_decode_size_in_one_launch():
     """The seven linears of a LLaMA-2-7B layer at T = 16: one launch, every output row against the oracle for three
     of them, all seven bit-identical to separate calls (which take the small-T kernel)."""

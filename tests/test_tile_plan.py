@@ -77,12 +77,14 @@ def test_multi_small_t_problems_share_a_launch_only_if_they_fill_the_chip():
     layer = lambda T: [(T, N, K) for K, N in LLAMA7B]
     for T in (1, 16, 128):
         assert launches(layer(T)) == 1                       # 200+ tiles for 74 pairs
-        assert launches(layer(T)[:3]) == 3                   # q/k/v alone: about 60 tiles, one small-T launch each
+        assert launches(layer(T)[:3]) == 1                   # q/k/v: too few tiles for the CTA pairs, but their 96
+                                                             # 128-channel tiles fit the device: one small-T launch
+        assert launches([(T, 1032, 512), (T, 520, 2048), (T + 1, 2048, 256)]) == 2     # another T: a launch of its own
         assert launches(layer(T)[4:6]) == 1                  # gate/up: 106 tiles
         assert launches(layer(T)[:1]) == 1
     # a small-T problem whose 128-channel tiles outnumber the SMs needs a quantizer launch of its own
     assert launches([(16, 19200, 80)]) == 2
-    # the same list on a (hypothetical) device with fewer resident pairs groups earlier
+    # the same list on a (hypothetical) device with fewer resident pairs fills the pairs and goes to them
     assert launches(layer(16)[:3], pairs=32) == 1
 
 
