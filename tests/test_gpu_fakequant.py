@@ -3,7 +3,7 @@ element by element on the same seeded bytes.
 
 Bars: y and dx bit-exact (16-bit patterns); the reduced scale gradient within
 1e-4 relative of the oracle's double-precision sum and bit-identical from run to
-run.  The tolerance on ds is the one the benchmark spec states; the arithmetic
+run.  The tolerance on ds is the stated bar of the library; the arithmetic
 (fp32 products, fp32 trees of 8, double accumulation) keeps the error near
 1e-7 * sum|g * term|.
 """
