@@ -45,7 +45,7 @@ L2_BYTES = 126 * 1024 * 1024
 INT8_OVER_BF16_NOMINAL = 2.0          # dense INT8 peak is twice the dense bf16 peak (4.5 vs 2.25 P-op/s nominal)
 # DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/ (T = 2048 workload only;
 # set to None whenever the kernel changes after its capture)
-NCU_TRAFFIC_FAKEQUANT = 533.2e6        # profiles/fakequant_kernel_llama7b_layer_T2048.md
+NCU_TRAFFIC_FAKEQUANT = 532.0e6        # profiles/fakequant_kernel_llama7b_layer_T2048.md
 NCU_TRAFFIC_GEMM = 671.0e6              # DRAM bytes of the step's one GEMM launch (profiles/w8a8_gemm_pair_kernel_T2048.md)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
