@@ -1,0 +1,419 @@
+// Small-T kernel (T <= 128): swapped operands, K split over a cluster, for one or several same-T problems.
+#pragma once
+
+#include "gemm_pair.cuh"
+
+namespace sasq {
+namespace {
+
+// ---------------------------------------------------------------------------
+// Small-T kernel (T <= 128: decode and short prompts).  The work is streaming W once from HBM, so the roles of the
+// operands are swapped: 128 rows of W are the M side of the MMA (every instruction consumes 4 KB of weights), the
+// T activation rows, padded to a multiple of 16, are the N side, and the accumulator tile in TMEM is
+// [128 output channels x T tokens].  To occupy the whole chip a cluster of S CTAs shares one 128-channel tile and
+// splits K; each CTA sends its partial accumulators through distributed shared memory to the CTA that owns the
+// channels (CTA r owns 128 / S of them), and after one cluster barrier every CTA adds the S partials of its channels
+// (int32: exact in any order), dequantises and stores them.
+//   warp 0      TMA producer: W tile (128 x 128 B) + int8 activation tile (TP x 128 B) per stage
+//   warp 1      MMA issuer
+//   warps 2..5  first the activation quantizer (Eq. 1 with the fixed factor, all CTAs share the T x K elements and
+//               publish through one counter; the producers load activation tiles only after it is complete, the
+//               weight tiles of the first stages are on their way by then), then the epilogue
+// ---------------------------------------------------------------------------
+constexpr int D_THREADS = 192;
+constexpr int D_W_BYTES = 128 * BK;          // weight tile of a stage
+constexpr int D_MAX_STAGES = 8;
+constexpr int D_RING_BYTES = 192 * 1024;     // stages x (weight tile + activation tile) fit in here
+
+struct DecodeTail {
+    uint64_t full[D_MAX_STAGES];
+    uint64_t empty[D_MAX_STAGES];
+    uint64_t acc_full;
+    uint32_t tmem_base;
+    volatile int abort_flag;
+    int is_last_cta;
+    float row_max[4];    // dynamic per-token factors: the four quantizer warps' maxima of the row in hand
+};
+
+// One launch may carry several independent problems with the same T (the q/k/v projections of a decode step, say):
+// the 128-channel tiles of all of them form one list of clusters, and every CTA helps to quantize every problem's x.
+constexpr int kMaxDecodeGroup = 8;
+struct DecodeProblem {
+    LinearParams lp;
+    const uint16_t* x;   // NULL: the codes in a_int8 were written by an earlier launch
+    uint8_t* a_int8;
+    int tile_begin;      // 128-channel tiles of the problems before this one
+};
+struct DecodeMaps {
+    CUtensorMap w[kMaxDecodeGroup], x[kMaxDecodeGroup];
+};
+struct DecodeParams {
+    int count;
+    DecodeProblem prob[kMaxDecodeGroup];
+    int tp;              // T rounded up to a multiple of 16: N of the MMA
+    int stages;
+    int split;           // CTAs per cluster = K slices
+    int n_tiles;         // 128-channel tiles of all problems
+    uint32_t tmem_cols;  // power of two >= max(32, tp)
+    int slots_offset;    // byte offset of the reduction slots in the CTA's shared memory: behind the stages, never
+                         // under them, because peers write there while this CTA may still be in its mainloop
+    bool quantize;       // the activation quantizer runs inside this launch
+    unsigned* ready;     // [count] per problem: 16-element items quantized and visible; zero at launch
+    unsigned* done;
+    float qn, qp;
+    float* row_scale_out;   // non-NULL: dynamic per-token factors, computed here (a CTA's four quantizer warps per
+                            // row) and written there; lp.row_scale points at the same array for the epilogue
+};
+
+constexpr int D_DYN_WORDS = 12;   // 128-bit words of a row a quantizer thread keeps in registers between the two passes
+
+__device__ __forceinline__ bool wait_bounded_d(uint64_t* bar, uint32_t parity, DecodeTail* tail, const LinearParams& p) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    int polls = 0;
+    while (!ptx::mbar_try_wait(bar, parity)) {
+        if (p.wait_limit <= 0 || (++polls & 63) == 0) {      // a zero limit gives up at the first unsuccessful poll
+            if (tail->abort_flag) return false;
+            if (clock64() - t0 > p.wait_limit) {
+                tail->abort_flag = 1;
+                atomicMax(p.status, (int)SASQ_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+template <bool BF>
+__global__ void __launch_bounds__(D_THREADS, 1)
+w8a8_decode_kernel(const __grid_constant__ DecodeMaps maps, const __grid_constant__ DecodeParams dp) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t* ring = smem_raw;
+    DecodeTail* tail = reinterpret_cast<DecodeTail*>(ring + D_RING_BYTES);
+    // the problem this cluster's tile belongs to
+    const int tile_all = blockIdx.x / dp.split;
+    int q_mine = 0;
+    while (q_mine + 1 < dp.count && tile_all >= dp.prob[q_mine + 1].tile_begin) ++q_mine;
+    const DecodeProblem& me = dp.prob[q_mine];
+    const LinearParams& p = me.lp;
+    const CUtensorMap* tmap_w = &maps.w[q_mine];
+    const CUtensorMap* tmap_x = &maps.x[q_mine];
+    if ((ptx::smem_u32(ring) & 1023u) != 0) {       // uniform over the grid: every CTA returns before any barrier
+        if (threadIdx.x == 0) atomicMax(p.status, (int)SASQ_ERR_CUDA);
+        return;
+    }
+    pdl_launch_dependents();
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int rank = (int)ptx::cluster_ctarank();
+    const int n_tile = tile_all - me.tile_begin;
+    const int n0 = n_tile * 128;
+    const int stage_bytes = D_W_BYTES + dp.tp * BK;
+    // this CTA's slice of the k-blocks
+    const int kb_begin = (int)(((long long)rank * p.k_blocks) / dp.split);
+    const int kb_end = (int)(((long long)(rank + 1) * p.k_blocks) / dp.split);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < dp.stages; ++s) {
+            ptx::mbar_init(&tail->full[s], 1);
+            ptx::mbar_init(&tail->empty[s], 1);
+        }
+        ptx::mbar_init(&tail->acc_full, 1);
+        tail->abort_flag = 0;
+        ptx::mbar_init_fence();
+        ptx::prefetch_tensormap(tmap_w);
+        ptx::prefetch_tensormap(tmap_x);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(&tail->tmem_base, dp.tmem_cols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = tail->tmem_base;
+    pdl_wait();                         // set-up done; from here on global memory of earlier kernels is used
+
+    // 16-element items the in-kernel quantizer has to publish (none if the activations came quantized)
+    const unsigned items_total = dp.quantize ? (unsigned)(((long long)p.T * p.K) >> 4) : 0u;   // of this CTA's problem
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (ptx::elect_one()) {
+            bool ok = true;
+            int stage = 0;
+            uint32_t phase = 0;
+            // weight tiles of the first stages go out at once; the activation tiles follow when every CTA has
+            // quantized its share of x
+            int early = kb_end - kb_begin < dp.stages ? kb_end - kb_begin : dp.stages;
+            for (int i = 0; i < early; ++i) {
+                ptx::mbar_arrive_expect_tx(&tail->full[i], (uint32_t)stage_bytes);
+                ptx::tma_load_2d(ring + (size_t)i * stage_bytes, tmap_w, &tail->full[i], (kb_begin + i) * BK, n0);
+            }
+            if (items_total != 0) {
+                const long long t0 = clock64();
+                int polls = 0;
+                for (;;) {
+                    unsigned v;
+                    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(dp.ready + q_mine) : "memory");
+                    if (v >= items_total) break;
+                    if (p.wait_limit <= 0 || (++polls & 15) == 0) {
+                        if (tail->abort_flag) { ok = false; break; }
+                        if (clock64() - t0 > p.wait_limit) {
+                            tail->abort_flag = 1;
+                            atomicMax(p.status, (int)SASQ_ERR_TIMEOUT);
+                            ok = false;
+                            break;
+                        }
+                    }
+                    __nanosleep(32);
+                }
+                asm volatile("fence.proxy.async.global;" ::: "memory");
+            }
+            for (int kb = kb_begin; kb < kb_end && ok; ++kb) {
+                uint8_t* w_dst = ring + (size_t)stage * stage_bytes;
+                if (kb - kb_begin >= early) {
+                    ok = wait_bounded_d(&tail->empty[stage], phase ^ 1u, tail, p);
+                    if (!ok) break;
+                    ptx::mbar_arrive_expect_tx(&tail->full[stage], (uint32_t)stage_bytes);
+                    ptx::tma_load_2d(w_dst, tmap_w, &tail->full[stage], kb * BK, n0);
+                }
+                ptx::tma_load_2d(w_dst + D_W_BYTES, tmap_x, &tail->full[stage], kb * BK, 0);
+                if (++stage == dp.stages) { stage = 0; phase ^= 1u; }
+            }
+            if (!ok) {      // copies in flight must land before the CTA's shared memory goes away
+                const long long t0 = clock64();
+                while (clock64() - t0 < (1LL << 22)) __nanosleep(1000);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (ptx::elect_one()) {
+            const uint32_t idesc = ptx::idesc_i8(128, dp.tp);
+            const uint64_t w_desc0 = ptx::smem_desc_k_major_sw128(ptx::smem_u32(ring));
+            const uint64_t x_desc0 = ptx::smem_desc_k_major_sw128(ptx::smem_u32(ring) + D_W_BYTES);
+            const uint32_t stage_step = (uint32_t)(stage_bytes >> 4);
+            int stage = 0;
+            uint32_t phase = 0;
+            uint32_t accumulate = 0;
+            bool ok = true;
+            for (int kb = kb_begin; kb < kb_end; ++kb) {
+                ok = wait_bounded_d(&tail->full[stage], phase, tail, p);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                const uint64_t w_desc = w_desc0 + (uint64_t)(stage * stage_step);
+                const uint64_t x_desc = x_desc0 + (uint64_t)(stage * stage_step);
+                ptx::mma_i8_ss(tmem_base, w_desc, x_desc, idesc, accumulate);
+                ptx::mma_i8_ss_acc(tmem_base, w_desc + 2, x_desc + 2, idesc);
+                ptx::mma_i8_ss_acc(tmem_base, w_desc + 4, x_desc + 4, idesc);
+                ptx::mma_i8_ss_acc(tmem_base, w_desc + 6, x_desc + 6, idesc);
+                accumulate = 1u;
+                ptx::mma_commit(&tail->empty[stage]);
+                if (++stage == dp.stages) { stage = 0; phase ^= 1u; }
+            }
+            if (ok) ptx::mma_commit(&tail->acc_full);       // also right for an empty slice: arrives at once
+        }
+        __syncwarp();
+    } else {
+        // ---------------- activation quantizer, then epilogue (warps 2..5) ----------------
+        const int et = threadIdx.x - 64;                       // 0..127
+        if (dp.quantize && dp.row_scale_out != nullptr) {
+            // Dynamic per-token quantization (Sec. 4.4, generation phase) inside the launch: the rows are dealt to
+            // the CTAs, and the 128 quantizer threads of a CTA take a row together.  The row's factor is its own
+            // max-based one, s_t = max_k |x[t,k]| / Qp (Eq. 1; an all-zero row takes s_t = 1).  Each thread keeps its
+            // words of the row in registers between the maximum and the quantization (rows longer than
+            // 128 x D_DYN_WORDS words read the rest a second time).
+            const int vec = p.K >> 3;
+            unsigned rows_done = 0;
+            for (int r = blockIdx.x; r < p.T; r += gridDim.x) {
+                const uint4* row = reinterpret_cast<const uint4*>(me.x) + (size_t)r * vec;
+                uint4 keep[D_DYN_WORDS];
+                float m = 0.0f;
+#pragma unroll
+                for (int u = 0; u < D_DYN_WORDS; ++u) {
+                    const int i = et + 128 * u;
+                    if (i < vec) {
+                        keep[u] = row[i];
+                        const uint32_t w4[4] = {keep[u].x, keep[u].y, keep[u].z, keep[u].w};
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const float2 f = widen2<BF>(w4[q]);
+                            m = fmaxf(m, fmaxf(fabsf(f.x), fabsf(f.y)));
+                        }
+                    }
+                }
+                for (int i = et + 128 * D_DYN_WORDS; i < vec; i += 128) {
+                    const uint4 v = row[i];
+                    const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float2 f = widen2<BF>(w4[q]);
+                        m = fmaxf(m, fmaxf(fabsf(f.x), fabsf(f.y)));
+                    }
+                }
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, off));
+                if (lane == 0) tail->row_max[warp - 2] = m;
+                asm volatile("bar.sync 3, 128;" ::: "memory");
+                m = fmaxf(fmaxf(tail->row_max[0], tail->row_max[1]), fmaxf(tail->row_max[2], tail->row_max[3]));
+                const float sc = m > 0.0f ? __fdiv_rn(m, dp.qp) : 1.0f;
+                const float inv = __fdiv_rn(1.0f, sc);
+                if (et == 0) dp.row_scale_out[r] = sc;
+                uint2* orow = reinterpret_cast<uint2*>(me.a_int8) + (size_t)r * vec;
+#pragma unroll
+                for (int u = 0; u < D_DYN_WORDS; ++u) {
+                    const int i = et + 128 * u;
+                    if (i < vec) orow[i] = quantize8<BF, false>(keep[u], inv, dp.qn, dp.qp);
+                }
+                for (int i = et + 128 * D_DYN_WORDS; i < vec; i += 128)
+                    orow[i] = quantize8<BF, false>(row[i], inv, dp.qn, dp.qp);
+                ++rows_done;
+                asm volatile("bar.sync 3, 128;" ::: "memory");      // row_max is free for the next row
+            }
+            asm volatile("fence.proxy.async.global;" ::: "memory");
+            __threadfence();
+            asm volatile("bar.sync 3, 128;" ::: "memory");          // every thread's codes are out and fenced
+            if (et == 0 && rows_done != 0) atomicAdd(dp.ready + q_mine, rows_done * (unsigned)(p.K >> 4));
+        } else if (dp.quantize) {
+            // every CTA takes its share of every problem's x, in problem order
+            for (int q = 0; q < dp.count; ++q) {
+                const DecodeProblem& pr = dp.prob[q];
+                const LinearParams& lp = pr.lp;
+                const bool one = lp.chan_inv == nullptr;                 // one static factor for the whole tensor
+                const float sxq = one ? __ldg(lp.x_scale) : 1.0f;
+                if (one && blockIdx.x == 0 && et == 0 && scale_is_bad(sxq)) atomicMax(lp.status, (int)SASQ_ERR_BAD_SCALE);
+                const float inv = __fdiv_rn(1.0f, sxq);
+                const uint4* src = reinterpret_cast<const uint4*>(pr.x);
+                uint4* dst = reinterpret_cast<uint4*>(pr.a_int8);
+                const unsigned items = (unsigned)(((long long)lp.T * lp.K) >> 4);
+                unsigned mine = 0;
+                for (unsigned i = blockIdx.x * 128u + (unsigned)et; i < items; i += gridDim.x * 128u) {
+                    const uint4 a = ld_stream16(src + 2 * (size_t)i), b = ld_stream16(src + 2 * (size_t)i + 1);
+                    uint2 lo, hi;
+                    if (lp.chan_inv != nullptr) {
+                        const float* ci = lp.chan_inv + 16 * (i % (unsigned)(lp.K >> 4));
+                        lo = quantize8_channels<BF>(a, ci, dp.qn, dp.qp);
+                        hi = quantize8_channels<BF>(b, ci + 8, dp.qn, dp.qp);
+                    } else {
+                        lo = quantize8<BF, false>(a, inv, dp.qn, dp.qp);
+                        hi = quantize8<BF, false>(b, inv, dp.qn, dp.qp);
+                    }
+                    dst[i] = make_uint4(lo.x, lo.y, hi.x, hi.y);
+                    ++mine;
+                }
+                asm volatile("fence.proxy.async.global;" ::: "memory");
+                __threadfence();
+                // one add per warp
+                for (int off = 16; off > 0; off >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, off);
+                if (lane == 0 && mine != 0) atomicAdd(dp.ready + q, mine);
+            }
+        } else if (blockIdx.x == 0 && et == 0 && p.row_scale == nullptr && p.chan_inv == nullptr &&
+                   scale_is_bad(__ldg(p.x_scale))) {
+            atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);             // codes from an earlier launch: check the factor
+        }
+
+        // epilogue part 1: this CTA's partial accumulators go from TMEM straight into the shared memory of the CTA
+        // that will reduce them (remote stores through distributed shared memory, into slots behind the pipeline stages).  CTA r
+        // owns channels [r * 128 / S, (r + 1) * 128 / S) of the tile and holds one slot per K slice:
+        // [S slots][128 / S channels][tp + 4 words]; rows tp + 4 words apart keep 128-bit accesses aligned and
+        // let eight consecutive rows cover all banks.
+        const int quad = warp & 3;                              // TMEM lane quadrant of this warp
+        const int pstride = dp.tp + 4;
+        const int rows = 128 / dp.split;
+        bool ok = wait_bounded_d(&tail->acc_full, 0u, tail, p);
+        ok = epilogue_all_ok(ok);
+        if (ok) {
+            ptx::tc_fence_after_sync();
+            const int n_local = quad * 32 + lane;
+            const int owner = n_local / rows;
+            const uint32_t local = ptx::smem_u32(ring) + (uint32_t)dp.slots_offset +
+                                   (uint32_t)((rank * rows + (n_local - owner * rows)) * pstride) * 4u;
+            const uint32_t dst = ptx::mapa_u32(local, (uint32_t)owner);
+            if (kb_end > kb_begin) {
+                const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
+                for (int c = 0; c < dp.tp; c += 16) {
+                    uint32_t v[16];
+                    ptx::tmem_ld_32x16(taddr + (uint32_t)c, v);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (uint32_t)(c + 4 * j) * 4u),
+                                     "r"(v[4 * j]), "r"(v[4 * j + 1]), "r"(v[4 * j + 2]), "r"(v[4 * j + 3]) : "memory");
+                }
+            } else {
+                for (int c = 0; c < dp.tp; c += 4)
+                    asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(dst + (uint32_t)c * 4u), "r"(0u)
+                                 : "memory");
+            }
+        }
+        ptx::tc_fence_before_sync();
+    }
+
+    // every CTA's partials are in their owner's shared memory after this barrier (or the launch has been abandoned:
+    // a role gave up after a bounded wait and the status word says so; the sums below are then garbage but every
+    // access stays in bounds).  Nobody touches another CTA's shared memory afterwards, so the CTAs may finish
+    // independently.
+    __syncthreads();
+    ptx::cluster_sync_all();
+
+    if (warp >= 2) {
+        // epilogue part 2: add the S slots of this CTA's channels, dequantise, store.  One work item = one channel
+        // x four consecutive tokens (one 128-bit read per slot); consecutive threads take consecutive channels so
+        // that the 16-bit stores of one token coalesce.
+        const int et = threadIdx.x - 64;
+        const int rows = 128 / dp.split;
+        const int pstride = dp.tp + 4;
+        const bool has_bias = p.bias != nullptr;
+        const bool per_row = p.row_scale != nullptr;
+        const float sx = (per_row || p.chan_inv != nullptr) ? 1.0f : __ldg(p.x_scale);
+        const int items = rows * (dp.tp >> 2);
+        const int32_t* slots = reinterpret_cast<const int32_t*>(ring + dp.slots_offset);
+        for (int it = et; it < items; it += 128) {
+            const int r_local = it % rows;
+            const int t0 = (it / rows) << 2;
+            const int n = n0 + rank * rows + r_local;
+            int32_t acc[4] = {0, 0, 0, 0};
+            for (int r = 0; r < dp.split; ++r) {
+                const int4 v = *reinterpret_cast<const int4*>(slots + (size_t)(r * rows + r_local) * pstride + t0);
+                acc[0] += v.x; acc[1] += v.y; acc[2] += v.z; acc[3] += v.w;
+            }
+            if (n < p.N) {
+                const float ws = __ldg(p.w_scale + n);
+                const float sc = __fmul_rn(sx, ws);
+                const float bv = has_bias ? widen1<BF>(__ldg(reinterpret_cast<const uint16_t*>(p.bias) + n)) : 0.0f;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int t = t0 + j;
+                    if (t < p.T) {
+                        // a plain load: in the dynamic mode other CTAs wrote the factors during this launch
+                        const float sct = per_row ? __fmul_rn(p.row_scale[t], ws) : sc;
+                        float f = __fmul_rn(__int2float_rn(acc[j]), sct);
+                        if (has_bias) f = __fadd_rn(f, bv);
+                        reinterpret_cast<uint16_t*>(p.y)[(size_t)t * p.N + n] = narrow1<BF>(f);
+                        if (p.acc_out != nullptr) p.acc_out[(size_t)t * p.N + n] = acc[j];
+                    }
+                }
+            }
+        }
+    }
+
+    // ---------------- teardown ----------------
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, dp.tmem_cols);
+    }
+    // the CTA that finishes last leaves the counters at zero for the next launch that draws them
+    if (dp.quantize && threadIdx.x == 0) {
+        if (atomicAdd(dp.done, 1u) == gridDim.x - 1) {
+            for (int q = 0; q < dp.count; ++q) dp.ready[q] = 0u;
+            *dp.done = 0u;
+        }
+    }
+}
+
+}  // namespace
+}  // namespace sasq
