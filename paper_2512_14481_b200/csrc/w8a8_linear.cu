@@ -667,7 +667,6 @@ int linear_impl(const void* x, const int8_t* w, const float* w_scale, const floa
     p.status = status;
     p.wait_limit = g_wait_limit.load(std::memory_order_relaxed);
     CUtensorMap tmap_a, tmap_w;
-    cudaError_t e;
     if (split > 0) {
         // small T: 128-channel tiles, K split over a cluster, activations quantized inside the kernel
         DecodeParams dp{};
