@@ -306,7 +306,7 @@ typedef struct sasq_linear_desc {
 /* Bytes of scratch sasq_static_w8a8_linear_multi needs for these problems (descs_host: HOST memory, count entries). */
 SASQ_API size_t sasq_static_w8a8_linear_multi_workspace(int count, const sasq_linear_desc_t* descs_host);
 
-/* Several independent static W8A8 linears (Sec. 4.4, Eq. 1 + Eq. 3, each exactly as sasq_static_w8a8_linear
+/* Several independent static W8A8 linears (Sec. 4.2 static factors, Eq. 1 + Eq. 2, each exactly as sasq_static_w8a8_linear
  * computes it: the results are bit-identical to `count` separate calls) submitted together, e.g. the q/k/v or the
  * gate/up projections of a decoder layer, which do not depend on one another.  Consecutive problems with T > 128 run
  * in ONE launch (up to 8 problems, 1024 256-row blocks and 80 MiB of int8 activation codes, i.e. sum of T x K,

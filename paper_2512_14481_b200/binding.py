@@ -18,7 +18,7 @@ __all__ = [
     "sasq_fakequant_fwd", "sasq_fakequant_bwd_workspace", "sasq_fakequant_bwd", "sasq_fakequant_fwd_bwd",
     "sasq_fakequant_multi_workspace", "sasq_fakequant_fwd_bwd_multi", "sasq_static_w8a8_linear_workspace",
     "sasq_static_w8a8_linear", "sasq_device_status", "QDesc", "sasq_absmax_scale_workspace", "sasq_absmax_scale",
-    "sasq_quantize_weight", "linear_launches", "sasq_fakequant_fwd_bwd_static", "sasq_static_w8a8_linear_tiles",
+    "sasq_quantize_weight", "sasq_fakequant_fwd_bwd_static", "sasq_static_w8a8_linear_tiles",
     "sasq_fakequant_per_channel_workspace", "sasq_fakequant_fwd_bwd_per_channel",
     "sasq_fakequant_fwd_bwd_ablation", "sasq_adamw_scales", "SASQ_FULL_OPERATOR", "SASQ_WITHOUT_ROUND",
     "SASQ_WITHOUT_CLAMP", "sasq_dynamic_w8a8_linear_workspace", "sasq_dynamic_w8a8_linear", "sasq_debug_set_wait_limit", "PcDesc", "sasq_fakequant_per_channel_multi_workspace",
@@ -34,13 +34,6 @@ SASQ_BF16 = 1
 SASQ_FULL_OPERATOR = 0
 SASQ_WITHOUT_ROUND = 1
 SASQ_WITHOUT_CLAMP = 2
-
-
-def linear_launches(T: int) -> int:
-    """Kernels one sasq_static_w8a8_linear call launches, for launch counting: one when the activation quantizer
-    runs inside the GEMM kernel (T <= 262144 and, for T <= 128, at most one 128-channel tile per SM), otherwise
-    the quantizer and the GEMM."""
-    return 1 if int(T) <= 262144 else 2
 
 
 _HERE = os.path.dirname(os.path.abspath(__file__))

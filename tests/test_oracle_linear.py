@@ -204,3 +204,87 @@ def test_dynamic_per_token_linear_against_numpy_on_small_inputs():
         assert np.array_equal(y[t], oracle.narrow(y32.astype(np.float32), oracle.BF16))
     assert not acc[3].any() and np.abs(np.clip(acc, None, None)).max() > 0
     assert np.abs(oracle.quantize_act(xb[0:1], oracle.BF16, float(s[0]), 8)).max() == 127     # the row maximum maps to Qp
+
+
+@pytest.mark.parametrize("tag", TAGS)
+def test_per_channel_linear_with_a_constant_factor_is_eq2_on_folded_weights(tag):
+    """Sec. 5.1 granularity (per-channel activations), static form: with the same factor c on every channel,
+    folding it into the frozen weights (w' = w*c, quantized per output channel) and then leaving the activation
+    factor out of the epilogue must give the per-tensor Eq. 2 result on the same folded weights with s_x = 1
+    in the epilogue but codes taken with c, bit for bit.  The per-tensor pieces are pinned above."""
+    rng = np.random.default_rng(21)
+    T, N, K = 6, 24, 96
+    x = to_bits(rng.standard_normal((T, K)) * 3, tag)
+    c = np.float32(0.043)
+    w = (rng.standard_normal((N, K)) * 0.02).astype(np.float32)
+    w_int, ws = oracle.quantize_weight((w * c).astype(np.float32))
+    y, acc = oracle.w8a8_linear_per_channel(x, tag, w_int, ws, np.full(K, c, np.float32))
+    codes = oracle.quantize_act(x, tag, float(c))                       # Eq. 1 with the common factor
+    acc_ref = oracle.int_gemm(codes, w_int)
+    assert np.array_equal(acc, acc_ref)
+    y_ref, _ = oracle.dequant(acc_ref, ws, 1.0, tag)
+    assert np.array_equal(y, y_ref)
+    # the per-tensor linear applies s_x in its epilogue: on the folded weights that would count c twice
+    y_twice, _, acc_t = oracle.w8a8_linear(x, tag, w_int, ws, float(c))
+    assert np.array_equal(acc_t, acc) and not np.array_equal(y_twice, y)
+
+
+@pytest.mark.parametrize("tag", TAGS)
+def test_per_channel_linear_against_exact_arithmetic_on_tiny_operands(tag):
+    """Eq. 1 per channel + Eq. 2 with the activation factors inside the weights, evaluated exactly: power-of-two
+    factors make every code an exact integer computed with Fractions, the accumulators are exact integer sums, and
+    with power-of-two w_scale the product acc*w_scale[n] is exact in fp32 (under 24 bits), so the output is that
+    rational number narrowed once (torch's conversion, an independent library routine).  A wrong output factor
+    (any activation factor left in the epilogue), a factor taken from the wrong channel or a transposed weight
+    fails here."""
+    from fractions import Fraction
+    rng = np.random.default_rng(22)
+    T, N, K = 4, 5, 6
+    s_vec = np.array([0.5, 0.25, 2.0, 1.0, 0.125, 4.0], np.float32)
+    # values on a 1/16 grid: exactly representable in both 16-bit types, with ties and clipping among them
+    xv = rng.integers(-64, 65, size=(T, K)) / 16.0
+    xv[0, 0] = 0.25          # 0.25/0.5 = 0.5  -> tie, rounds to 0
+    xv[0, 1] = 0.375         # 0.375/0.25 = 1.5 -> tie, rounds to 2
+    xv[1, 4] = 40.0          # 40/0.125 = 320 -> clips to 127
+    xv[2, 4] = -40.0         # clips to -128
+    x = to_bits(xv, tag)
+    w_int = rng.integers(-5, 6, size=(N, K)).astype(np.int8)
+    ws = np.array([1.0, 0.5, 2.0, 0.25, 4.0], np.float32)
+    y, acc = oracle.w8a8_linear_per_channel(x, tag, w_int, ws, s_vec)
+
+    def rne(fr):
+        fl = fr.numerator // fr.denominator
+        rem = fr - fl
+        if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and fl % 2 == 1):
+            return fl + 1
+        return fl
+
+    codes = [[min(max(rne(Fraction(float(xv[t, k])) / Fraction(float(s_vec[k]))), -128), 127) for k in range(K)]
+             for t in range(T)]
+    assert codes[0][0] == 0 and codes[0][1] == 2 and codes[1][4] == 127 and codes[2][4] == -128
+    for t in range(T):
+        for n in range(N):
+            a = sum(codes[t][k] * int(w_int[n, k]) for k in range(K))
+            assert int(acc[t, n]) == a
+            exact = Fraction(a) * Fraction(float(ws[n]))
+            assert abs(a) < 2 ** 24 and Fraction(float(exact)) == exact       # exact in fp32 and in a double
+            want = torch.tensor([float(exact)], dtype=torch.float32).to(TDT[tag]).to(torch.float64).item()
+            assert float(from_bits(y[t:t + 1, n:n + 1], tag)[0, 0]) == want
+
+
+def test_per_channel_linear_planted_mistakes_fail_the_pins():
+    """What the two pins above catch, shown on the CPU: an activation factor left in the epilogue, and the
+    factors applied to the wrong channels."""
+    rng = np.random.default_rng(23)
+    T, N, K = 3, 4, 8
+    tag = BF16
+    s_vec = (2.0 ** rng.integers(-3, 3, K)).astype(np.float32)
+    x = to_bits(rng.integers(-64, 65, size=(T, K)) / 16.0, tag)
+    w_int = rng.integers(-5, 6, size=(N, K)).astype(np.int8)
+    ws = np.ones(N, np.float32)
+    y, acc = oracle.w8a8_linear_per_channel(x, tag, w_int, ws, s_vec)
+    _, codes = oracle.fakequant_fwd_per_channel(x, tag, s_vec)
+    y_bad, _ = oracle.dequant(oracle.int_gemm(codes.astype(np.int8), w_int), ws, 0.5, tag)
+    assert not np.array_equal(y_bad, y)
+    _, acc_rev = oracle.w8a8_linear_per_channel(x, tag, w_int, ws, s_vec[::-1].copy())
+    assert not np.array_equal(acc_rev, acc)
