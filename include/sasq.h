@@ -384,14 +384,15 @@ SASQ_API int sasq_adamw_scales(float* scales_dev, const float* grad_scales_dev, 
 
 /* Concurrency of the linear entry points.  When the activation quantizer runs inside the GEMM launch (every static
  * linear with T <= 262144 whose tiles fit the device), CTAs of that launch wait for codes that other CTAs of the
- * same launch write, so the launch is sized to be resident as a whole -- on an otherwise free device.  If kernels on
- * OTHER streams hold SMs meanwhile, the missing CTAs start when those kernels end; two such launches that overlap on
- * different streams can each hold the SMs the other is waiting for, in which case their bounded waits give up after
- * about a second with SASQ_ERR_TIMEOUT (outputs unspecified, nothing hangs).  Callers that run these entry points
- * on several streams of one device at once, or beside long-running kernels, switch this on: the launches are then
- * made as co-operative grids, which the driver starts only when every CTA can be resident.  It costs the overlap of
- * a launch's set-up with its predecessor's tail, about 2 us per launch on a B200.  on: non-zero / zero; applies to
- * launches made afterwards, process-wide; returns the previous setting (default 0).  The paper has no counterpart. */
+ * same launch write, so all of its CTAs must be resident together.  By default (on != 0) these launches are
+ * therefore made as co-operative grids, which the driver starts only when every CTA can be resident: linears may
+ * then run on several streams of one device at once, or beside other kernels, and merely queue behind one another.
+ * A caller that submits all of its linears on ONE stream of an otherwise idle device may switch this off
+ * (on == 0): plain launches let a launch's set-up overlap its predecessor's tail, about 2 us per launch on a B200.
+ * With it off, two such launches that overlap on different streams can each hold the SMs the other is waiting for;
+ * their bounded waits then give up after about a second with SASQ_ERR_TIMEOUT in the status word (outputs
+ * unspecified, nothing hangs).  Applies to launches made afterwards, process-wide; returns the previous setting.
+ * The paper has no counterpart. */
 SASQ_API int sasq_set_gang_launch(int on);
 
 /* Test hook.  Every wait inside the GEMM kernels (on an mbarrier, on the activation quantizer's counters) gives up
@@ -400,6 +401,18 @@ SASQ_API int sasq_set_gang_launch(int on);
  * it.  Returns the previous limit.  Applies to launches made afterwards.  sasq_device_status clears the library's
  * internal counters when it reports a timeout, so the next call starts clean. */
 SASQ_API long long sasq_debug_set_wait_limit(long long cycles);
+
+/* Measurement aid (the paper has no counterpart; Sec. 2 only names integer GEMM kernels as usable).  Runs, on every
+ * resident CTA pair of the device, `mma_per_pair` (>= 32, rounded down to a multiple of 32) back-to-back
+ * tcgen05.mma.cta_group::2.kind::i8 instructions of shape 256 x n_cols x 32 (n_cols a multiple of 32 in [32, 256])
+ * on pseudo-random int8 operands held in shared memory: the instruction the static W8A8 linear is built from, with no loads and no
+ * epilogue around it.  Synchronises `stream`.  Writes to HOST memory: *ops_per_second_host = integer operations
+ * (2 per multiply-accumulate) of the whole device over the CUDA-event time of the launch, and *mac_per_clk_sm_host
+ * = multiply-accumulates per SM clock cycle per SM on the slowest pair.  A few ms of MMAs give the burst rate, a
+ * second or more the rate under the power cap.  Allocates nothing.  Errors: SASQ_ERR_INVALID_ARG,
+ * SASQ_ERR_UNSUPPORTED (not sm_100), SASQ_ERR_TIMEOUT (a bounded wait gave up), SASQ_ERR_CUDA. */
+SASQ_API int sasq_debug_int8_issue_rate(int mma_per_pair, int n_cols, double* ops_per_second_host,
+                                        double* mac_per_clk_sm_host, void* stream);
 
 /* Synchronises `stream`, returns the sticky device status word of the current
  * device (SASQ_OK, SASQ_ERR_BAD_SCALE or SASQ_ERR_TIMEOUT) and clears it. */

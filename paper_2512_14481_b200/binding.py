@@ -26,7 +26,8 @@ __all__ = [
     "sasq_static_w8a8_linear_per_channel", "sasq_static_w8a8_linear_grouped_workspace",
     "sasq_static_w8a8_linear_grouped", "sasq_fakequant_linear_fp_weights_workspace",
     "sasq_fakequant_linear_fp_weights", "sasq_absmax_scale_per_channel", "sasq_running_mean", "LinearDesc", "sasq_static_w8a8_linear_multi_workspace",
-    "sasq_static_w8a8_linear_multi", "sasq_static_w8a8_linear_multi_launches", "sasq_set_gang_launch", "LinearProblems", "QuantTensors",
+    "sasq_static_w8a8_linear_multi", "sasq_static_w8a8_linear_multi_launches", "sasq_set_gang_launch",
+    "sasq_debug_int8_issue_rate", "LinearProblems", "QuantTensors",
 ]
 
 SASQ_F16 = 0
@@ -189,9 +190,19 @@ def _stream(stream) -> int:
     return s.cuda_stream
 
 
+# SASQ_DEBUG_STATUS=1 in the environment: every call through this binding also synchronises and reads the sticky
+# device status word, so that a device-detected problem (a bad factor, a bounded wait that gave up) raises at the
+# call that caused it instead of waiting for the caller's next sasq_device_status().  For tests and debugging only.
+_DEBUG_STATUS = os.environ.get("SASQ_DEBUG_STATUS", "0") not in ("", "0")
+
+
 def _check(status: int, where: str):
     if status != 0:
         raise SasqError(status, where)
+    if _DEBUG_STATUS:
+        dev_status = int(load_library().sasq_device_status(_stream(None)))
+        if dev_status != 0:
+            raise SasqError(dev_status, where + " (device status)")
 
 
 def _nbytes(t) -> int:
@@ -585,9 +596,22 @@ def sasq_debug_set_wait_limit(cycles: int) -> int:
     return int(load_library().sasq_debug_set_wait_limit(int(cycles)))
 
 
+def sasq_debug_int8_issue_rate(mma_per_pair: int, n_cols: int = 256, stream=None):
+    """Measurement aid: back-to-back int8 tensor-core instructions of the GEMM's shape on every CTA pair.
+    Returns (integer operations per second of the device, multiply-accumulates per clock per SM)."""
+    L = load_library()
+    L.sasq_debug_int8_issue_rate.restype = ctypes.c_int
+    L.sasq_debug_int8_issue_rate.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_double),
+                                             ctypes.POINTER(ctypes.c_double), ctypes.c_void_p]
+    ops, mac = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    _check(L.sasq_debug_int8_issue_rate(int(mma_per_pair), int(n_cols), ctypes.byref(ops), ctypes.byref(mac),
+                                        _stream(stream)), "sasq_debug_int8_issue_rate")
+    return float(ops.value), float(mac.value)
+
+
 def sasq_set_gang_launch(on: bool) -> bool:
-    """Launch the linears whose CTAs wait on one another as co-operative grids (for callers that overlap them on
-    several streams); returns the previous setting."""
+    """Launch the linears whose CTAs wait on one another as co-operative grids (the default; safe with several
+    streams).  A caller that keeps all linears on one stream may pass False; returns the previous setting."""
     L = load_library()
     L.sasq_set_gang_launch.restype = ctypes.c_int
     L.sasq_set_gang_launch.argtypes = [ctypes.c_int]

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsasq_b200.so")
-SOURCES = ["api.cu", "fakequant.cu", "fakequant_per_channel.cu", "w8a8_linear.cu", "calibrate.cu"]
+SOURCES = ["api.cu", "fakequant.cu", "fakequant_per_channel.cu", "w8a8_linear.cu", "calibrate.cu", "peak_probe.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden",

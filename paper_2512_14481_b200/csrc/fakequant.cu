@@ -29,7 +29,10 @@ constexpr int kThreads = 256;
 constexpr int kUnroll = 2;             // 128-bit vectors of x (and of g) in flight per thread
 constexpr int kUnrollFwdOnly = 4;      // the forward alone loads half as much per vector: keep as many bytes in flight
 constexpr int kBlocksPerSM = 4;
-constexpr int kLoadHint = 1;
+#ifndef SASQ_FQ_LOAD_HINT
+#define SASQ_FQ_LOAD_HINT 1
+#endif
+constexpr int kLoadHint = SASQ_FQ_LOAD_HINT;
 constexpr int kStoreHint = 1;
 
 int* status_word_ptr() {
@@ -45,22 +48,37 @@ int* status_word_ptr() {
 }
 
 // Ticket counters of the second reduction stage.  They are zero when the library is loaded and every launch
-// leaves the one it used at zero again.  Launches draw them round-robin, so two launches share a counter only if
-// more than kTicketSlots launches of this library were executing at the same time, which no GPU does.
+// leaves the one it used at zero again.  Launches made directly draw them round-robin, so two of them share a counter
+// only if more than kTicketSlots launches of this library were executing at the same time, which no GPU does.  A
+// launch that is being captured into a CUDA graph keeps its counter's address for every replay, at times the library
+// does not see: it gets a counter of its own from a second pool that is never handed out twice (kCaptureTickets
+// captured launches per process), so a replay can overlap other launches of the library on other streams.
 constexpr unsigned kTicketSlots = 256;
-static __device__ unsigned g_tickets[kTicketSlots];
+constexpr unsigned kCaptureTickets = 4096;
+static __device__ unsigned g_tickets[kTicketSlots + kCaptureTickets];
 
-unsigned* next_ticket() {
+// SASQ_OK and *ticket, or SASQ_ERR_UNSUPPORTED when a captured launch finds the capture pool used up
+int next_ticket(cudaStream_t st, unsigned** ticket) {
     static unsigned* base[64] = {nullptr};
     static std::atomic<unsigned> next{0};
+    static std::atomic<unsigned> capture_next{0};
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SASQ_ERR_CUDA;
     if (base[dev] == nullptr) {
         unsigned* p = nullptr;
-        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_tickets) != cudaSuccess) return nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_tickets) != cudaSuccess) return SASQ_ERR_CUDA;
         base[dev] = p;
     }
-    return base[dev] + (next.fetch_add(1u, std::memory_order_relaxed) % kTicketSlots);
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &capturing) != cudaSuccess) return SASQ_ERR_CUDA;
+    if (capturing != cudaStreamCaptureStatusNone) {
+        const unsigned at = capture_next.fetch_add(1u, std::memory_order_relaxed);
+        if (at >= kCaptureTickets) return SASQ_ERR_UNSUPPORTED;
+        *ticket = base[dev] + kTicketSlots + at;
+        return SASQ_OK;
+    }
+    *ticket = base[dev] + (next.fetch_add(1u, std::memory_order_relaxed) % kTicketSlots);
+    return SASQ_OK;
 }
 
 template <bool BF, bool FWD, bool BWD, int VARIANT = 0>
@@ -109,15 +127,19 @@ int run_multi(const sasq_qdesc_t* descs, int n_tensors, const float* scales_dev,
     if (dt != SASQ_F16 && dt != SASQ_BF16) return SASQ_ERR_INVALID_ARG;
     if (n_tensors == 0) return SASQ_OK;
 
-    const bool fwd = descs[0].y != nullptr;
-    const bool bwd = descs[0].grad_y != nullptr;
+    // the first descriptor that holds elements says which passes run; empty ones (numel == 0) may leave every
+    // pointer NULL and are skipped by the kernel
+    int lead = 0;
+    while (lead + 1 < n_tensors && descs[lead].numel == 0) ++lead;
+    const bool fwd = descs[lead].y != nullptr;
+    const bool bwd = descs[lead].grad_y != nullptr;
     long long max_numel = 0;
     for (int i = 0; i < n_tensors; ++i) {
         const sasq_qdesc_t& d = descs[i];
         if (d.numel < 0 || d.reserved != 0) return SASQ_ERR_INVALID_ARG;
         if (d.scale_index < 0 || d.scale_index >= n_scales) return SASQ_ERR_INVALID_ARG;
-        if ((d.y != nullptr) != fwd || (d.grad_y != nullptr) != bwd) return SASQ_ERR_INVALID_ARG;
-        if ((d.grad_y != nullptr) != (d.grad_x != nullptr)) return SASQ_ERR_INVALID_ARG;
+        if (d.numel > 0 && ((d.y != nullptr) != fwd || (d.grad_y != nullptr) != bwd)) return SASQ_ERR_INVALID_ARG;
+        if (d.numel > 0 && (d.grad_y != nullptr) != (d.grad_x != nullptr)) return SASQ_ERR_INVALID_ARG;
         if (d.numel > 0 && d.x == nullptr) return SASQ_ERR_INVALID_ARG;
         if (!aligned16(d.x) || !aligned16(d.y) || !aligned16(d.grad_y) || !aligned16(d.grad_x))
             return SASQ_ERR_INVALID_ARG;
@@ -162,8 +184,8 @@ int run_multi(const sasq_qdesc_t* descs, int n_tensors, const float* scales_dev,
         p.status = status;
         p.grad_scales = grad_scales_dev;
         if (bwd) {
-            p.ticket = next_ticket();
-            if (p.ticket == nullptr) return SASQ_ERR_CUDA;
+            const int ticket_rc = next_ticket(st, &p.ticket);
+            if (ticket_rc != SASQ_OK) return ticket_rc;
         }
         cudaError_t e = (dt == SASQ_BF16) ? launch_variant<true>(variant, fwd, bwd, p, grid, st)
                                           : launch_variant<false>(variant, fwd, bwd, p, grid, st);
@@ -273,8 +295,8 @@ int sasq_fakequant_fwd_bwd_static(const void* x, const void* grad_y, void* y, vo
     p.status = status;
     p.grad_scales = grad_scale_dev;
     p.accumulate_mask = accumulate ? 1u : 0u;
-    p.ticket = next_ticket();
-    if (p.ticket == nullptr) return SASQ_ERR_CUDA;
+    const int ticket_rc = next_ticket(st, &p.ticket);
+    if (ticket_rc != SASQ_OK) return ticket_rc;
     const cudaError_t e = (dt == SASQ_BF16) ? launch_mode<true>(true, true, p, grid, st)
                                             : launch_mode<false>(true, true, p, grid, st);
     if (e != cudaSuccess) return SASQ_ERR_CUDA;

@@ -103,9 +103,14 @@ __device__ __forceinline__ uint4 load16(const uint4* p) {
     } else if constexpr (HINT == 1) {
         asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                      : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    } else {
+    } else if constexpr (HINT == 2) {
         asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];"
                      : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    } else {
+        // streaming, not kept in L1, through the coherent path: valid when the launch also stores to these addresses
+        // (y may alias x and grad_x may alias grad_y)
+        asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
     }
     return v;
 }

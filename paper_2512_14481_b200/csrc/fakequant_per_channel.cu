@@ -215,7 +215,10 @@ int pc_run(const sasq_pcdesc_t* descs, int n, int accumulate, int dt, int bits, 
     if (bits < 2 || bits > 8 || (dt != SASQ_F16 && dt != SASQ_BF16)) return SASQ_ERR_INVALID_ARG;
     if (n == 0) return SASQ_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const bool fwd = descs[0].y != nullptr, bwd = descs[0].grad_y != nullptr;
+    // the first descriptor that has rows says which passes run; tensors without rows may leave the data pointers NULL
+    int lead = 0;
+    while (lead + 1 < n && descs[lead].T == 0) ++lead;
+    const bool fwd = descs[lead].y != nullptr, bwd = descs[lead].grad_y != nullptr;
     long long total_elems = 0, total_k = 0;
     int live = 0;
     for (int i = 0; i < n; ++i) {
@@ -226,7 +229,7 @@ int pc_run(const sasq_pcdesc_t* descs, int n, int accumulate, int dt, int bits, 
             if ((d.y != nullptr) != fwd || (d.grad_y != nullptr) != bwd) return SASQ_ERR_INVALID_ARG;
             if ((d.grad_y != nullptr) != (d.grad_x != nullptr) || d.x == nullptr) return SASQ_ERR_INVALID_ARG;
         }
-        if (bwd && d.grad_scales == nullptr) return SASQ_ERR_INVALID_ARG;
+        if (bwd && d.T > 0 && d.grad_scales == nullptr) return SASQ_ERR_INVALID_ARG;
         if (!aligned16(d.x) || !aligned16(d.grad_y) || !aligned16(d.y) || !aligned16(d.grad_x) || !aligned16(d.scales))
             return SASQ_ERR_INVALID_ARG;
         if (d.T > 0) { total_elems += d.T * d.K; total_k += d.K; ++live; }

@@ -24,7 +24,9 @@ constexpr int EPI_THREADS = 128;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr long long kWaitLimit = 1LL << 31;   // clock cycles a single wait may take (about a second)
 std::atomic<long long> g_wait_limit{kWaitLimit};   // what launches use; tests shorten it to see the give-up path
-std::atomic<int> g_gang_launch{0};                 // launch the kernels whose CTAs wait on one another as co-operative grids
+// launch the kernels whose CTAs wait on one another as co-operative grids (the safe default: such a launch starts only
+// when all of its CTAs can be resident; a caller that keeps every linear on one stream may switch it off)
+std::atomic<int> g_gang_launch{1};
 
 struct SharedTail {
     uint64_t full[STAGES];

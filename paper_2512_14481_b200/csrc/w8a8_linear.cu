@@ -132,41 +132,66 @@ bool make_tmap_out(CUtensorMap* m, const void* base, long long T, long long N, i
 }
 
 // Counters of the in-kernel activation quantizer.  They are zero when the library is loaded and every launch leaves
-// the set it used at zero again; launches draw the sets round-robin, so two launches share one only if more than
-// kReadySlots launches of this kernel were running at the same time.
+// the set it used at zero again.  Launches made directly draw the sets round-robin, so two of them share one only if
+// more than kReadySlots launches of this kernel were running at the same time.  A launch that is being captured into
+// a CUDA graph is different: its counters' address is frozen into the graph and used again by every replay, at
+// times the library does not see.  Such a launch gets counters of its own from a second pool that is never handed
+// out twice (a bump allocator; kCaptureCounters counters per process), so a replay can overlap launches made
+// directly, or other graphs, on other streams without sharing a counter with them.
 static __device__ unsigned g_a_ready[kReadySlots][kMaxRowBlocks];
 static __device__ unsigned g_a_done[kReadySlots];
+constexpr unsigned kCaptureCounters = 1u << 16;
+static __device__ unsigned g_a_capture[kCaptureCounters];
 
 }  // namespace
 
 void linear_reset_counters(cudaStream_t st) {
-    void *r = nullptr, *d = nullptr;
-    if (cudaGetSymbolAddress(&r, g_a_ready) == cudaSuccess && cudaGetSymbolAddress(&d, g_a_done) == cudaSuccess) {
+    void *r = nullptr, *d = nullptr, *c = nullptr;
+    if (cudaGetSymbolAddress(&r, g_a_ready) == cudaSuccess && cudaGetSymbolAddress(&d, g_a_done) == cudaSuccess &&
+        cudaGetSymbolAddress(&c, g_a_capture) == cudaSuccess) {
         cudaMemsetAsync(r, 0, sizeof(unsigned) * kReadySlots * kMaxRowBlocks, st);
         cudaMemsetAsync(d, 0, sizeof(unsigned) * kReadySlots, st);
+        cudaMemsetAsync(c, 0, sizeof(unsigned) * kCaptureCounters, st);
         cudaStreamSynchronize(st);
     }
 }
 
 namespace {
 
-bool next_ready_slot(unsigned** ready, unsigned** done) {
+// `count` readiness counters and one completion counter for a launch on `st`.  SASQ_ERR_UNSUPPORTED when a captured
+// launch finds the capture pool used up.
+int next_ready_slot(cudaStream_t st, int count, unsigned** ready, unsigned** done) {
     static unsigned* ready_base[64] = {nullptr};
     static unsigned* done_base[64] = {nullptr};
+    static unsigned* capture_base[64] = {nullptr};
     static std::atomic<unsigned> next{0};
+    static std::atomic<unsigned> capture_next{0};
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SASQ_ERR_CUDA;
     if (ready_base[dev] == nullptr) {
-        unsigned *r = nullptr, *d = nullptr;
-        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&r), g_a_ready) != cudaSuccess) return false;
-        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&d), g_a_done) != cudaSuccess) return false;
+        unsigned *r = nullptr, *d = nullptr, *c = nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&r), g_a_ready) != cudaSuccess) return SASQ_ERR_CUDA;
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&d), g_a_done) != cudaSuccess) return SASQ_ERR_CUDA;
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&c), g_a_capture) != cudaSuccess) return SASQ_ERR_CUDA;
         done_base[dev] = d;
+        capture_base[dev] = c;
         ready_base[dev] = r;
+    }
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &capturing) != cudaSuccess) return SASQ_ERR_CUDA;
+    if (capturing != cudaStreamCaptureStatusNone) {
+        if (count < 0 || count > kMaxRowBlocks) return SASQ_ERR_UNSUPPORTED;
+        const unsigned want = (unsigned)count + 1u;
+        const unsigned at = capture_next.fetch_add(want, std::memory_order_relaxed);
+        if (at > kCaptureCounters || at + want > kCaptureCounters) return SASQ_ERR_UNSUPPORTED;
+        *ready = capture_base[dev] + at;
+        *done = capture_base[dev] + at + count;
+        return SASQ_OK;
     }
     const unsigned slot = next.fetch_add(1u, std::memory_order_relaxed) % kReadySlots;
     *ready = ready_base[dev] + (size_t)slot * kMaxRowBlocks;
     *done = done_base[dev] + slot;
-    return true;
+    return SASQ_OK;
 }
 
 // Number of CTA pairs that can be resident at once (one pair per TPC); also opts the kernel in to its shared memory.
@@ -459,7 +484,10 @@ int launch_decode_group(DecodeMaps& maps, DecodeParams& dp, int T, int split, bo
     dp.split = split;
     dp.tmem_cols = 32;
     while ((int)dp.tmem_cols < dp.tp) dp.tmem_cols <<= 1;
-    if (dp.quantize && !next_ready_slot(&dp.ready, &dp.done)) return SASQ_ERR_CUDA;
+    if (dp.quantize) {
+        const int rc = next_ready_slot(st, dp.count, &dp.ready, &dp.done);
+        if (rc != SASQ_OK) return rc;
+    }
     for (int q = 0; q < dp.count; ++q)
         if (!make_tmap(&maps.x[q], dp.prob[q].a_int8, T, dp.prob[q].lp.K, dp.tp)) return SASQ_ERR_CUDA;
     cudaLaunchConfig_t cfg{};
@@ -706,9 +734,10 @@ int linear_impl(const void* x, const int8_t* w, const float* w_scale, const floa
         if (in_kernel_quantizer) {
             pp.x = static_cast<const uint16_t*>(x);
             pp.a_int8 = a_int8;
-            if (!next_ready_slot(&gp.ready, &gp.done)) return SASQ_ERR_CUDA;
-            pp.ready = gp.ready;
             gp.ready_count = pp.pair_m_blocks;
+            const int slot_rc = next_ready_slot(st, gp.ready_count, &gp.ready, &gp.done);
+            if (slot_rc != SASQ_OK) return slot_rc;
+            pp.ready = gp.ready;
             gp.num_chunks = (T * (K >> 3) + CONV_CHUNK - 1) / CONV_CHUNK;
         }
         if (!make_tmap(&maps.a[0], a_int8, T, K, 128) || !make_tmap(&maps.w[0], w, N, K, pp.w_box_rows) ||
@@ -832,13 +861,16 @@ int sasq_static_w8a8_linear_multi(int count, const sasq_linear_desc_t* descs_hos
             gp.count = q + 1;
         }
         if (gp.count == 0) return SASQ_OK;
-        if (!next_ready_slot(&gp.ready, &gp.done)) return SASQ_ERR_CUDA;
         int off = 0;
+        for (int q = 0; q < gp.count; ++q) off += gp.prob[q].pair_m_blocks;
+        gp.ready_count = off;
+        const int slot_rc = next_ready_slot(st, gp.ready_count, &gp.ready, &gp.done);
+        if (slot_rc != SASQ_OK) return slot_rc;
+        off = 0;
         for (int q = 0; q < gp.count; ++q) {
             gp.prob[q].ready = gp.ready + off;
             off += gp.prob[q].pair_m_blocks;
         }
-        gp.ready_count = off;
         deal_tiles_by_cost(&gp, pairs);
         return launch_pair_group(maps, gp, pairs, bf, st, small_layout);
     };

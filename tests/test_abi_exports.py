@@ -67,6 +67,12 @@ def test_host_side_argument_errors_launch_nothing():
     d[0] = P.QDesc(a, a, a, a, 8, 0, 0)
     d[1] = P.QDesc(a, None, a, None, 8, 0, 0)
     assert lib.sasq_fakequant_fwd_bwd_multi(d, 2, a, a, 2, 0, 1, 8, a, 1 << 20, None) == INVALID
+    # an empty first tensor (numel 0, no pointers) does not decide which passes run: the list is valid and the call
+    # gets as far as the workspace check
+    d[0] = P.QDesc(None, None, None, None, 0, 0, 0)
+    d[1] = P.QDesc(a, a, a, a, 8, 1, 0)
+    assert lib.sasq_fakequant_fwd_bwd_multi(d, 2, a, a, 2, 0, 1, 8, None, 0, None) == WORKSPACE
+    d[0] = P.QDesc(a, a, a, a, 8, 0, 0)
     d[1] = P.QDesc(a, a, a, a, 8, 0, 1)     # reserved must be 0
     assert lib.sasq_fakequant_fwd_bwd_multi(d, 2, a, a, 2, 0, 1, 8, a, 1 << 20, None) == INVALID
 

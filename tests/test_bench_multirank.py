@@ -45,10 +45,24 @@ def test_two_cpu_ranks_take_the_slowest_time_and_sum_the_work():
     assert bench.max_over_ranks([1.0, 2.0], None, "cpu") == [1.0, 2.0]
 
 
-def test_workload_constants_match_the_llama2_7b_layer():
+def test_workload_constants_match_the_llama2_7b_shapes():
     sys.path.insert(0, ROOT)
     import bench
     import sasq_workloads as W
     elems = 2048 * (6 * 4096 + 11008)
-    assert bench.quantizer_bytes() == 8 * elems == 583_008_256
-    assert bench.linear_ops() == 2 * 2048 * sum(K * N for _, K, N in W.LLAMA2_7B_LINEARS)
+    assert bench.quantizer_bytes(2048) == 8 * elems == 583_008_256
+    assert bench.linear_ops(2048) == 2 * 2048 * sum(K * N for _, K, N in W.LLAMA2_7B_LINEARS) == 828_928_688_128
+    # the full stack: 32 layers over 8 x 2048 tokens, 224 quantizers
+    assert bench.quantizer_bytes(16384, 32) == 32 * 8 * 16384 * (6 * 4096 + 11008)
+    assert bench.linear_ops(16384, 32) == 32 * 8 * bench.linear_ops(2048)
+    assert "T16384" in bench.workload_name(32, 16384) and "32_layers" in bench.workload_name(32, 16384)
+
+
+def test_tensor_peak_follows_the_length_of_the_timed_region():
+    sys.path.insert(0, ROOT)
+    import bench
+    peaks = {"bf16_tflops": 1600.0, "bf16_tflops_sustained": 1400.0}
+    assert bench.tensor_peak_for(0.0075, peaks, "measured")[0] == 3200.0        # a burst of a few ms
+    assert bench.tensor_peak_for(2.5, peaks, "measured")[0] == 2800.0           # seconds under the power cap
+    assert "burst" in bench.tensor_peak_for(0.0075, peaks, "measured")[1]
+    assert "sustained" in bench.tensor_peak_for(2.5, peaks, "measured")[1]

@@ -1,9 +1,10 @@
 """Linears submitted from two streams at once.
 
-Kernels with the activation quantizer inside have CTAs that wait for other CTAs of the same launch.  With
-sasq_set_gang_launch(1) such launches are co-operative grids, which the driver starts only when all their CTAs can be
-resident, so launches that overlap on different streams cannot starve each other.  The test checks that the setting
-changes no bit of any result and that interleaved launches on two streams all complete with the right outputs.
+Kernels with the activation quantizer inside have CTAs that wait for other CTAs of the same launch.  By default
+such launches are co-operative grids, which the driver starts only when all their CTAs can be resident, so launches
+that overlap on different streams cannot starve each other; sasq_set_gang_launch(0) makes them plain launches for
+callers that keep to one stream.  The test checks that the setting changes no bit of any result and that interleaved
+launches on two streams (default setting) all complete with the right outputs.
 """
 import pytest
 import torch
@@ -33,12 +34,15 @@ def run(pr, stream=None):
 
 def test_gang_launch_changes_no_result_and_streams_can_overlap():
     cases = [make(700, 1032, 512, 31), make(16, 4096, 1024, 32), make(2048, 4096, 1024, 33), make(1, 2048, 4096, 34)]
-    want = [run(pr) for pr in cases]
-    torch.cuda.synchronize()
-    assert P.sasq_device_status() == 0
-    previous = P.sasq_set_gang_launch(True)
+    previous = P.sasq_set_gang_launch(False)          # plain launches, one stream: the reference results
+    assert previous is True                           # co-operative launches are the default
     try:
-        assert previous is False
+        want = [run(pr) for pr in cases]
+        torch.cuda.synchronize()
+        assert P.sasq_device_status() == 0
+    finally:
+        P.sasq_set_gang_launch(True)
+    try:
         for pr, ref in zip(cases, want):                       # same bits with co-operative launches
             assert torch.equal(run(pr).view(torch.int16), ref.view(torch.int16))
         s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
@@ -58,4 +62,4 @@ def test_gang_launch_changes_no_result_and_streams_can_overlap():
         for i, y in outs:
             assert torch.equal(y.view(torch.int16), want[i].view(torch.int16)), i
     finally:
-        P.sasq_set_gang_launch(False)
+        P.sasq_set_gang_launch(True)
