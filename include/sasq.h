@@ -219,7 +219,13 @@ SASQ_API size_t sasq_static_w8a8_linear_workspace(int64_t T, int64_t N, int64_t 
  * Sec. 3).  y: [T, N] of `dt`.  acc_out: [T, N] int32 or NULL; when given, the
  * raw accumulators are also written (parity / debugging).
  * Constraints: K % 16 == 0, N % 8 == 0, K <= 131072 (int32 cannot overflow),
- * bits in [2, 8]; otherwise SASQ_ERR_UNSUPPORTED. */
+ * bits in [2, 8]; otherwise SASQ_ERR_UNSUPPORTED.
+ * The weights are frozen (Sec. 4.2): `w` is read as soon as the kernel is resident, which, for a call that follows
+ * another call of this library on the same stream, can be before that earlier kernel has finished.  No call of this
+ * library writes int8 weights on that fast path (sasq_quantize_weight does not let its successor start early), so
+ * this matters only to a caller that hands `w` a buffer some other SASQ call on the stream is still writing as
+ * its 16-bit output: do not.  x, x_scale_dev, w_scale, bias and y are touched only after every earlier kernel of
+ * the stream has completed. */
 SASQ_API int sasq_static_w8a8_linear(const void* x, const int8_t* w, const float* w_scale, const float* x_scale_dev,
                             const void* bias, void* y, int32_t* acc_out, int64_t T, int64_t N, int64_t K,
                             int dt, int bits, void* workspace, size_t ws_bytes, void* stream);

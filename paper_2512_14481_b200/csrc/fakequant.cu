@@ -29,8 +29,10 @@ constexpr int kThreads = 256;
 constexpr int kUnroll = 2;             // 128-bit vectors of x (and of g) in flight per thread
 constexpr int kUnrollFwdOnly = 4;      // the forward alone loads half as much per vector: keep as many bytes in flight
 constexpr int kBlocksPerSM = 4;
+// streaming loads through the coherent path (hint 3): y may alias x and grad_x may alias grad_y, so the launch may
+// store to the addresses it loads from, which rules out the non-coherent (.nc) form; measured at the same speed
 #ifndef SASQ_FQ_LOAD_HINT
-#define SASQ_FQ_LOAD_HINT 1
+#define SASQ_FQ_LOAD_HINT 3
 #endif
 constexpr int kLoadHint = SASQ_FQ_LOAD_HINT;
 constexpr int kStoreHint = 1;

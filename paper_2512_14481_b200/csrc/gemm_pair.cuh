@@ -46,8 +46,22 @@ constexpr int P_MAX_STAGES = P_SMALL_STAGES > P_STAGES ? P_SMALL_STAGES : P_STAG
 constexpr int P_NUM_THREADS = 448;       // 14 warps: producer, MMA issuer, 4 epilogue, 8 activation quantizer
 constexpr int CONV_THREADS = 256;
 constexpr int CONV_WARPS = CONV_THREADS / 32;
-constexpr int CONV_ITEMS = 16;           // 8-element items per lane and chunk: 16 128-bit loads in flight per lane
-constexpr int CONV_CHUNK = 32 * CONV_ITEMS;   // items per chunk: one warp, 4096 elements
+// 8-element items per lane and chunk = 128-bit loads in flight per lane.  A launch cannot issue an MMA before the row
+// blocks of its first wave of tiles are quantized and published, and a chunk is one serial chain (load, convert,
+// store, fence, publish): the chunk is sized so that the first round of chunks over all workers of the grid just
+// covers those row blocks.
+#ifndef SASQ_CONV_ITEMS
+#define SASQ_CONV_ITEMS 10
+#endif
+constexpr int CONV_ITEMS = SASQ_CONV_ITEMS;
+constexpr int CONV_CHUNK = 32 * CONV_ITEMS;   // items per chunk (one warp)
+// The four epilogue warps of a CTA have nothing to drain until the first tile's accumulators are complete: they take
+// part in the first rounds of the chunk list as workers 8..11 of their CTA.
+#ifndef SASQ_EPI_CONV_ROUNDS
+#define SASQ_EPI_CONV_ROUNDS 1
+#endif
+constexpr int EPI_CONV_ROUNDS = SASQ_EPI_CONV_ROUNDS;
+constexpr int CONV_HEAD_WORKERS = CONV_WARPS + 4;
 constexpr int kMaxRowBlocks = 1024;      // 256-row blocks the in-kernel quantizer can publish (T <= 262144)
 constexpr int kReadySlots = 32;          // concurrently running launches that can each own a set of counters
 
@@ -129,6 +143,9 @@ struct TileWalk {
     __device__ __forceinline__ bool more() const { return at < end; }
     __device__ __forceinline__ void next() { at += step; }
     __device__ __forceinline__ int tile(const GroupParams& gp) const { return list ? (int)gp.tile_list[at] : at; }
+    __device__ __forceinline__ bool is_last() const { return at + step >= end; }
+    // tiles still to come, this one included
+    __device__ __forceinline__ int remaining() const { return at < end ? (end - at + step - 1) / step : 0; }
 };
 // the problem tile g belongs to
 __device__ __forceinline__ int problem_of(const GroupParams& gp, int g) {
@@ -205,6 +222,9 @@ __device__ __forceinline__ uint4 ld_stream16(const uint4* p) {
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;
 }
+// (L2 policies for this traffic were measured and not kept: storing the codes with an evict-last policy brings the
+// DRAM traffic of a T = 16384 launch down from 1.23 to 1.09 times its algorithmic bytes, but the launch is not bound
+// by DRAM and the sustained rate fell by 2 %; loading x with evict-first changed nothing.)
 
 // ---- in-kernel activation quantizer: one chunk = 32 lanes x CONV_ITEMS items of 8 elements, contiguous in x ----
 struct ConvJob {
@@ -254,9 +274,9 @@ __device__ __forceinline__ void conv_store(const ConvJob& j, long long c, int la
 // every lane's stores visible at GPU scope (and to the TMA unit), then one add per row block the chunk touches
 __device__ __forceinline__ void conv_publish(const ConvJob& j, long long c, int lane) {
     asm volatile("fence.proxy.async.global;" ::: "memory");
-    __threadfence();
     __syncwarp();
     if (lane == 0) {
+        __threadfence();        // cumulative: orders the stores of every lane (observed through the warp barrier)
         const long long first = c * CONV_CHUNK;
         const long long end = (first + CONV_CHUNK < j.total) ? first + CONV_CHUNK : j.total;
         long long i = first;
@@ -309,6 +329,241 @@ __device__ __forceinline__ bool wait_bounded_pair(uint64_t* bar, uint32_t parity
     return true;
 }
 
+// The chunk list of a launch (all problems, in problem order) as one worker of a CTA walks it.  Rounds below
+// EPI_CONV_ROUNDS are dealt over 12 workers per CTA (the quantizer warps, slots 0..7, and the epilogue warps, slots
+// 8..11), later rounds over the 8 quantizer warps; within a round the workers of the grid take consecutive chunks, so
+// the row blocks become ready in the order the tiles need them.  Every warp runs its own load -> quantize -> store ->
+// fence -> publish chain with CONV_ITEMS 128-bit loads in flight per lane.
+template <bool BF>
+__device__ __forceinline__ void conv_rounds(const GroupParams& gp, int slot, bool epilogue_warp, int lane) {
+    const long long grid = (long long)gridDim.x;
+    const long long head = (long long)EPI_CONV_ROUNDS * grid * CONV_HEAD_WORKERS;
+    ConvJob job{};
+    int q = 0, job_q = -1;
+    for (int r = 0;; ++r) {
+        long long c;
+        if (r < EPI_CONV_ROUNDS) {
+            c = ((long long)r * grid + blockIdx.x) * CONV_HEAD_WORKERS + slot;
+        } else {
+            if (epilogue_warp) break;
+            c = head + ((long long)(r - EPI_CONV_ROUNDS) * grid + blockIdx.x) * CONV_WARPS + slot;
+        }
+        if (c >= gp.num_chunks) break;          // c grows with r
+        while (q + 1 < gp.count && c >= gp.prob[q + 1].chunk_begin) ++q;
+        if (q != job_q) {
+            const PairParams& pp = gp.prob[q];
+            const LinearParams& p = pp.lp;
+            job.src = reinterpret_cast<const uint4*>(pp.x);
+            job.dst = reinterpret_cast<uint2*>(pp.a_int8);
+            job.ready = pp.ready;
+            job.total = (long long)p.T * (p.K >> 3);
+            job.items_per_block = (long long)PBM * (p.K >> 3);
+            job.chan_inv = p.chan_inv;
+            job.vec_per_row = (unsigned)(p.K >> 3);
+            job.qn = pp.qn;
+            job.qp = pp.qp;
+            job.eight = pp.qp == 127.0f;
+        }
+        const long long lc = c - gp.prob[q].chunk_begin;
+        uint4 v[CONV_ITEMS];
+        conv_load(job, lc, lane, v);
+        if (q != job_q) {       // the factor is fetched with the chunk's loads already in flight
+            const LinearParams& p = gp.prob[q].lp;
+            job.inv = p.chan_inv == nullptr ? __fdiv_rn(1.0f, __ldg(p.x_scale)) : 0.0f;
+            job_q = q;
+        }
+        conv_store<BF>(job, lc, lane, v);
+        conv_publish(job, lc, lane);
+    }
+}
+
+// ---- epilogue of (a share of) one tile by one warp ----
+// The warp owns 32 rows (one TMEM lane quadrant of its CTA).  The tile's columns are cut into units of 64 columns
+// (whole 128-byte lines) and, where the width is not a multiple of 64, trailing units of 16 columns; worker w of
+// `workers` warps that share the quadrant takes units w, w + workers, ...  Per unit: TMEM -> registers -> dequantise
+// -> the warp's 128-byte- (32-byte-) swizzled staging tile -> one TMA store (rows >= T and columns >= N are clipped
+// by the tensor map).
+struct EpiTile {
+    const LinearParams* p;
+    const CUtensorMap* y64;
+    const CUtensorMap* y16;
+    uint64_t policy;
+    uint32_t taddr;         // TMEM address of the quadrant's lanes, first column of the accumulator buffer
+    int n0, bn, row0;
+    const float* scale;     // [bn] staged s_x * s_w[n] (or s_w[n] with per-row factors)
+    const float* bias;      // [bn] staged bias
+};
+
+// Dequantisation of 8 adjacent accumulators of one row into four packed 16-bit pairs.  PLAIN: one static factor per
+// tensor and no bias, the hot case: convert, one multiply, narrow.  Otherwise the per-row factor and the bias are
+// applied as the flags say.  The epilogue is bound by the instructions it issues (a tile has 32768 values per CTA;
+// the int -> float conversions alone keep the SM's 16-lane conversion pipe busy for 2048 cycles), so the hot case
+// carries none it does not need.  (Converting on the integer and FMA pipes instead -- split the value in two
+// 16-bit halves, make each a float through the mantissa of a constant, join them with one fused multiply-add --
+// is exact too but costs six issue slots per value: measured 1 to 2 % slower.)
+template <bool BF, bool PLAIN>
+__device__ __forceinline__ uint4 dequant8(const uint32_t* v, const float* s8, const float* b8, bool per_row,
+                                          float s_row, bool has_bias) {
+    uint32_t o[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        float f0, f1;
+        if constexpr (PLAIN) {
+            f0 = __fmul_rn(__int2float_rn((int)v[2 * q]), s8[2 * q]);
+            f1 = __fmul_rn(__int2float_rn((int)v[2 * q + 1]), s8[2 * q + 1]);
+        } else {
+            f0 = __fmul_rn(__int2float_rn((int)v[2 * q]), out_scale(per_row, s_row, s8[2 * q]));
+            f1 = __fmul_rn(__int2float_rn((int)v[2 * q + 1]), out_scale(per_row, s_row, s8[2 * q + 1]));
+            if (has_bias) {
+                f0 = __fadd_rn(f0, b8[2 * q]);
+                f1 = __fadd_rn(f1, b8[2 * q + 1]);
+            }
+        }
+        o[q] = narrow2<BF>(f0, f1);
+    }
+    return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+// 16 adjacent columns of the warp's 32 rows: factors (and bias) read from the staged arrays first, then two
+// 16-byte pieces written to the staging tile (`piece0`, `piece0 + 1` of a row of `row_bytes` bytes, swizzled) and,
+// when asked for, the raw accumulators to acc_out.
+template <bool BF, bool PLAIN>
+__device__ __forceinline__ void dequant16_to_stage(const uint32_t* v, const float* sc, const float* bi, bool per_row,
+                                                   float s_row, bool has_bias, uint8_t* sbuf, int lane, int row_bytes,
+                                                   int piece0, int32_t* acc_dst, bool acc_ok0, bool acc_ok1) {
+    // the loads of a piece before its store: the compiler cannot tell the staged factors from the staging tile and
+    // keeps every load behind the store before it
+    const int sw = row_bytes == 128 ? (lane & 7) : ((lane >> 2) & 1);
+#pragma unroll
+    for (int h8 = 0; h8 < 2; ++h8) {
+        float s8[8], b8[8];
+        const float4 f0 = *reinterpret_cast<const float4*>(sc + 8 * h8);
+        const float4 f1 = *reinterpret_cast<const float4*>(sc + 8 * h8 + 4);
+        s8[0] = f0.x; s8[1] = f0.y; s8[2] = f0.z; s8[3] = f0.w; s8[4] = f1.x; s8[5] = f1.y; s8[6] = f1.z; s8[7] = f1.w;
+        if constexpr (!PLAIN) {
+            if (has_bias) {
+                const float4 c0 = *reinterpret_cast<const float4*>(bi + 8 * h8);
+                const float4 c1 = *reinterpret_cast<const float4*>(bi + 8 * h8 + 4);
+                b8[0] = c0.x; b8[1] = c0.y; b8[2] = c0.z; b8[3] = c0.w;
+                b8[4] = c1.x; b8[5] = c1.y; b8[6] = c1.z; b8[7] = c1.w;
+            }
+        }
+        const uint4 o = dequant8<BF, PLAIN>(v + 8 * h8, s8, b8, per_row, s_row, has_bias);
+        *reinterpret_cast<uint4*>(sbuf + lane * row_bytes + (((piece0 + h8) ^ sw) << 4)) = o;
+        if (acc_dst != nullptr && (h8 == 0 ? acc_ok0 : acc_ok1)) {
+            int32_t* a = acc_dst + 8 * h8;
+            *reinterpret_cast<uint4*>(a) = make_uint4(v[8 * h8], v[8 * h8 + 1], v[8 * h8 + 2], v[8 * h8 + 3]);
+            *reinterpret_cast<uint4*>(a + 4) = make_uint4(v[8 * h8 + 4], v[8 * h8 + 5], v[8 * h8 + 6], v[8 * h8 + 7]);
+        }
+    }
+}
+
+// copy_out: the staging tile is copied to global memory by the warp itself (128-bit loads from shared memory, 128-bit
+// stores, eight lanes per 128-byte row) instead of by a TMA store.  A TMA store has to have read the staging tile
+// before the CTA may leave (about a microsecond after it is issued, measured), which nothing hides after the last
+// tile of a pair; plain stores are simply complete when the grid is.
+template <bool BF>
+__device__ __forceinline__ void epilogue_units(const EpiTile& t, uint8_t* my_stage, unsigned& out_flip, int lane,
+                                               int worker, int workers, bool copy_out) {
+    const LinearParams& p = *t.p;
+    const bool per_row = p.row_scale != nullptr;
+    const bool has_bias = p.bias != nullptr;
+    const bool plain = !per_row && !has_bias;
+    const int row = t.row0 + lane;
+    const bool row_ok = row < p.T;
+    const float s_row = (per_row && row_ok) ? __ldg(p.row_scale + row) : 1.0f;
+    int32_t* arow = (p.acc_out && row_ok) ? p.acc_out + (size_t)row * p.N + t.n0 : nullptr;
+    uint16_t* y = reinterpret_cast<uint16_t*>(p.y);
+    const int n64 = t.bn >> 6;
+    const int units = n64 + ((t.bn & 63) >> 4);
+#pragma unroll 1
+    for (int u = worker; u < units; u += workers) {
+        uint8_t* sbuf = my_stage + (size_t)(out_flip & 1) * P_OUT_BUF_BYTES;
+        if (lane == 0) ptx::bulk_wait_group_read<1>();      // the store that used this buffer has read it
+        __syncwarp();
+        if (u < n64) {
+            const int c = u << 6;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                uint32_t v[32];
+                ptx::tmem_ld_32x32(t.taddr + (uint32_t)(c + 32 * h), v);
+                ptx::tmem_ld_wait();
+#pragma unroll
+                for (int g16 = 0; g16 < 32; g16 += 16) {
+                    const int col = c + 32 * h + g16;               // first of these 16 columns, within the tile
+                    const bool ok0 = (t.n0 + col) < p.N, ok1 = (t.n0 + col + 8) < p.N;
+                    if (plain)
+                        dequant16_to_stage<BF, true>(v + g16, t.scale + col, t.bias + col, false, 1.0f, false, sbuf, lane,
+                                                     128, (col & 63) >> 3, arow ? arow + col : nullptr, ok0, ok1);
+                    else
+                        dequant16_to_stage<BF, false>(v + g16, t.scale + col, t.bias + col, per_row, s_row, has_bias,
+                                                      sbuf, lane, 128, (col & 63) >> 3, arow ? arow + col : nullptr,
+                                                      ok0, ok1);
+                }
+            }
+            if (copy_out) {
+                __syncwarp();
+                const int piece = lane & 7;
+                const int col = t.n0 + c + piece * 8;           // N is a multiple of 8: a piece is inside or outside
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = (lane >> 3) + 4 * i;
+                    const uint4 w = *reinterpret_cast<const uint4*>(sbuf + r * 128 + ((piece ^ (r & 7)) << 4));
+                    if (t.row0 + r < p.T && col < p.N)
+                        *reinterpret_cast<uint4*>(y + (size_t)(t.row0 + r) * p.N + col) = w;
+                }
+            } else {
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    ptx::tma_store_2d_hint(t.y64, sbuf, t.n0 + c, t.row0, t.policy);
+                    ptx::bulk_commit_group();
+                }
+            }
+        } else {                            // 16 columns: 32-byte rows, 32-byte swizzle
+            const int c = (n64 << 6) + ((u - n64) << 4);
+            uint32_t v[16];
+            ptx::tmem_ld_32x16(t.taddr + (uint32_t)c, v);
+            ptx::tmem_ld_wait();
+            const bool ok0 = (t.n0 + c) < p.N, ok1 = (t.n0 + c + 8) < p.N;
+            if (plain)
+                dequant16_to_stage<BF, true>(v, t.scale + c, t.bias + c, false, 1.0f, false, sbuf, lane, 32, 0,
+                                             arow ? arow + c : nullptr, ok0, ok1);
+            else
+                dequant16_to_stage<BF, false>(v, t.scale + c, t.bias + c, per_row, s_row, has_bias, sbuf, lane, 32, 0,
+                                              arow ? arow + c : nullptr, ok0, ok1);
+            if (copy_out) {
+                __syncwarp();
+                const int piece = lane & 1;
+                const int col = t.n0 + c + piece * 8;
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const int r = (lane >> 1) + 16 * i;
+                    const uint4 w = *reinterpret_cast<const uint4*>(sbuf + r * 32 + ((piece ^ ((r >> 2) & 1)) << 4));
+                    if (t.row0 + r < p.T && col < p.N)
+                        *reinterpret_cast<uint4*>(y + (size_t)(t.row0 + r) * p.N + col) = w;
+                }
+            } else {
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    ptx::tma_store_2d_hint(t.y16, sbuf, t.n0 + c, t.row0, t.policy);
+                    ptx::bulk_commit_group();
+                }
+            }
+        }
+        if (copy_out) __syncwarp();         // the staging tile has been read before the next unit overwrites it
+        ++out_flip;
+    }
+}
+
+// The last tile of a pair is drained with nothing left to overlap it: the tensor pipe of the pair idles meanwhile, and
+// so does every other SM that is already done.  The eight quantizer warps, long finished, share that tile's epilogue:
+// each TMEM lane quadrant is served by its epilogue warp (worker 0) and the two quantizer warps whose index has the
+// same value mod 4 (workers 1 and 2).  They run the very loop the epilogue warps run (one copy of the code, already
+// in the instruction cache from the tiles before: a second, cold copy took longer to fetch than the work it does).
+constexpr int LAST_TILE_WORKERS = 3;
+
 template <bool BF, bool SMALL>
 __global__ void __launch_bounds__(P_NUM_THREADS, 1)
 w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_constant__ GroupParams gp) {
@@ -360,7 +615,10 @@ w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
     ptx::cluster_sync_all();            // both CTAs' barriers exist before anyone signals across the pair
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = tail->tmem_base;
-    pdl_wait();                         // set-up done; from here on global memory of earlier kernels is used
+    // Set-up done.  From here on memory that earlier kernels of the stream may have written (x, the factors) or may
+    // still be reading (y, the workspace) is used.  The producer warp waits later: the frozen weights depend on no
+    // earlier kernel, so it first puts the W halves of its first stages in flight.
+    if (warp != 0) pdl_wait();
 
     const int pair_id = blockIdx.x >> 1;
     const int num_pairs = gridDim.x >> 1;
@@ -372,6 +630,7 @@ w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
             uint32_t phase = 0;
             bool ok = true;
             int ready_blk = -1, ready_q = -1;
+            bool dep_waited = false;
             for (TileWalk walk(gp, pair_id, num_pairs); walk.more() && ok; walk.next()) {
                 const int g = walk.tile(gp);
                 const int q = problem_of(gp, g);
@@ -407,12 +666,14 @@ w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
                         ++kb_a;
                         if (++st == STAGES) { st = 0; ph ^= 1u; }
                     }
+                    if (!dep_waited) { pdl_wait(); dep_waited = true; }
                     ok = wait_rows_ready(pp.ready + m_blk, need, tail, p);
                     if (!ok) break;
                     asm volatile("fence.proxy.async.global;" ::: "memory");
                     ready_blk = m_blk;
                     ready_q = q;
                 }
+                if (!dep_waited) { pdl_wait(); dep_waited = true; }       // codes written by an earlier launch
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
                     uint8_t* w_dst = tiles + (size_t)stage * STAGE_BYTES;
                     // Only the leader arms the barrier (with the bytes of both CTAs); the partner's copies
@@ -480,191 +741,99 @@ w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
             }
         }
         __syncwarp();
-    } else if (warp >= 6) {
-        // ---------------- activation quantizer (warps 6..13 of both CTAs) ----------------
-        // x is taken as a flat run of T * K / 8 items of 8 elements, cut into chunks of 4096 elements that are
-        // dealt round-robin over all quantizer warps of the grid in address order, so the row blocks become ready
-        // in the order the tiles need them.  Every warp runs its own load -> quantize -> store -> fence -> publish
-        // pipeline with 16 128-bit loads in flight per lane; the warps drift apart, which keeps DRAM busy while
-        // some of them wait for their stores to be acknowledged.
-        // With several problems in the launch their chunks form one list, in problem order.
-        {
-            const int cw = warp - (P_NUM_THREADS - CONV_THREADS) / 32;          // 0..7
-            const long long stride = (long long)gridDim.x * CONV_WARPS;
-            ConvJob job{};
-            int q = 0, job_q = -1;
-            for (long long c = (long long)blockIdx.x * CONV_WARPS + cw; c < gp.num_chunks; c += stride) {
-                while (q + 1 < gp.count && c >= gp.prob[q + 1].chunk_begin) ++q;
-                if (q != job_q) {
-                    const PairParams& pp = gp.prob[q];
-                    const LinearParams& p = pp.lp;
-                    job.src = reinterpret_cast<const uint4*>(pp.x);
-                    job.dst = reinterpret_cast<uint2*>(pp.a_int8);
-                    job.ready = pp.ready;
-                    job.total = (long long)p.T * (p.K >> 3);
-                    job.items_per_block = (long long)PBM * (p.K >> 3);
-                    job.chan_inv = p.chan_inv;
-                    job.vec_per_row = (unsigned)(p.K >> 3);
-                    job.inv = p.chan_inv == nullptr ? __fdiv_rn(1.0f, __ldg(p.x_scale)) : 0.0f;
-                    job.qn = pp.qn;
-                    job.qp = pp.qp;
-                    job.eight = pp.qp == 127.0f;
-                    job_q = q;
-                }
-                const long long lc = c - gp.prob[q].chunk_begin;
-                uint4 v[CONV_ITEMS];
-                conv_load(job, lc, lane, v);
-                conv_store<BF>(job, lc, lane, v);
-                conv_publish(job, lc, lane);
-            }
-        }
     } else {
-        // ---------------- epilogue (warps 2..5 of both CTAs) ----------------
-        const int quad = warp & 3;
-        const int et = threadIdx.x - 64;
-        if (blockIdx.x == 0 && et < gp.count) {          // one thread per problem checks its static factor
+        // ---------------- warps 2..5: epilogue; warps 6..13: activation quantizer (both CTAs) ----------------
+        // All twelve first quantize: x is taken as a flat run of T * K / 8 items of 8 elements, cut into chunks that
+        // are dealt over the workers of the grid in address order (conv_rounds; the epilogue warps, which have
+        // nothing to drain until the first accumulators are complete, only take part in the first rounds).  With
+        // several problems in the launch their chunks form one list, in problem order.
+        // Then the epilogue warps drain every tile of the pair, overlapped with the MMAs of the next one, and the
+        // quantizer warps join them for the last tile.
+        const bool helper = warp >= 6;
+        const int cw = warp - (P_NUM_THREADS - CONV_THREADS) / 32;          // 0..7 for the quantizer warps
+        const int quad = warp & 3;                                           // TMEM lane quadrant of this warp
+        const int et = threadIdx.x - 64;                                     // 0..127 for the epilogue warps
+        if (!helper && blockIdx.x == 0 && et < gp.count) {          // one thread per problem checks its static factor
             const LinearParams& pe = gp.prob[et].lp;
             if (pe.row_scale == nullptr && pe.chan_inv == nullptr && scale_is_bad(__ldg(pe.x_scale)))
                 atomicMax(pe.status, (int)SASQ_ERR_BAD_SCALE);
         }
+        if (gp.num_chunks != 0) conv_rounds<BF>(gp, helper ? cw : CONV_WARPS + (warp - 2), !helper, lane);
+
         // The outputs are not read again by this launch: their lines should leave L2 first, during the launch (whose
         // DRAM interface is mostly idle), instead of staying behind dirty and being written back under the next kernel.
         const uint64_t y_policy = ptx::l2_policy_evict_first();
+        const int worker = helper ? 1 + (cw >> 2) : 0;
+        // staging tiles for the TMA stores: the epilogue warps have their own; the quantizer warps, which only work
+        // on the last tile, take the first pipeline stages (the accumulators of the last tile are complete by then,
+        // so every MMA of the pair has read its operands and no load is in flight)
+        uint8_t* my_stage = helper ? tiles + (size_t)cw * (2 * P_OUT_BUF_BYTES)
+                                   : out_stage + (size_t)quad * (2 * P_OUT_BUF_BYTES);
         bool ok = true;
         int it = 0;
         unsigned out_flip = 0;
-        for (TileWalk walk(gp, pair_id, num_pairs); walk.more() && ok; walk.next(), ++it) {
+        bool helpers_released = false;
+        TileWalk walk(gp, pair_id, num_pairs);
+        const bool any_tile = walk.more();
+        for (; walk.more() && ok; walk.next(), ++it) {
+            const bool last = walk.is_last();
+            if (helper && !last) continue;
             const int g = walk.tile(gp);
             const int q = problem_of(gp, g);
             const PairParams& pp = gp.prob[q];
             const LinearParams& p = pp.lp;
-            const CUtensorMap* tmap_y64 = &maps.y64[q];
-            const CUtensorMap* tmap_y16 = &maps.y16[q];
-            const bool per_row = p.row_scale != nullptr;
-            const bool one_factor = !per_row && p.chan_inv == nullptr;       // one static factor for the whole tensor
-            const float sx = one_factor ? __ldg(p.x_scale) : 1.0f;
-            const bool has_bias = p.bias != nullptr;
             const int tile = g - pp.tile_begin;
             const int m_blk = tile / pp.n_tiles;
-            int n0, bn;
-            pair_tile_cols(pp, tile - m_blk * pp.n_tiles, &n0, &bn);
+            EpiTile t;
+            pair_tile_cols(pp, tile - m_blk * pp.n_tiles, &t.n0, &t.bn);
             const int buf = it & 1;
             const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            for (int j = et; j < bn; j += EPI_THREADS) {
-                const int n = n0 + j;
-                tail->scale[j] = (n < p.N) ? __fmul_rn(sx, __ldg(p.w_scale + n)) : 0.0f;
-                if (has_bias)
-                    tail->bias[j] = (n < p.N) ? widen1<BF>(__ldg(reinterpret_cast<const uint16_t*>(p.bias) + n)) : 0.0f;
+            if (!helper) {
+                const bool one_factor = p.row_scale == nullptr && p.chan_inv == nullptr;   // one factor for the tensor
+                const float sx = one_factor ? __ldg(p.x_scale) : 1.0f;
+                const bool has_bias = p.bias != nullptr;
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                for (int j = et; j < t.bn; j += EPI_THREADS) {
+                    const int n = t.n0 + j;
+                    tail->scale[j] = (n < p.N) ? __fmul_rn(sx, __ldg(p.w_scale + n)) : 0.0f;
+                    if (has_bias)
+                        tail->bias[j] =
+                            (n < p.N) ? widen1<BF>(__ldg(reinterpret_cast<const uint16_t*>(p.bias) + n)) : 0.0f;
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (last) {         // the factors of the last tile are staged: the quantizer warps may read them
+                    asm volatile("bar.arrive 3, 384;" ::: "memory");
+                    helpers_released = true;
+                }
+            } else {
+                // the epilogue warps arrive here once they have staged the last tile's factors (or have given up)
+                asm volatile("bar.sync 3, 384;" ::: "memory");
+                ok = tail->abort_flag == 0;
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-
-            ok = wait_bounded_pair(&tail->tmem_full[buf], acc_phase, tail, p);
-            ok = epilogue_all_ok(ok);
+            if (ok) ok = wait_bounded_pair(&tail->tmem_full[buf], acc_phase, tail, p);
+            if (!helper) ok = epilogue_all_ok(ok);
             if (!ok) break;
             ptx::tc_fence_after_sync();
 
-            // Each warp owns 32 rows.  64 columns at a time: TMEM -> registers -> dequantise -> this warp's
-            // 128-byte-swizzled staging tile -> one TMA store (whole 128-byte lines; rows >= T and columns >= N
-            // are clipped by the tensor map).  A tile width that is not a multiple of 64 ends in 16-column pieces.
-            const int row0 = m_blk * PBM + (int)rank * 128 + quad * 32;
-            const int row = row0 + lane;
-            const bool row_ok = row < p.T;
-            const float s_row = (per_row && row_ok) ? __ldg(p.row_scale + row) : 1.0f;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * 256);
-            int32_t* arow = p.acc_out ? p.acc_out + (size_t)row * p.N + n0 : nullptr;
-            uint8_t* my_stage = out_stage + (size_t)quad * 2 * P_OUT_BUF_BYTES;
-            int c = 0;
-#pragma unroll 1
-            for (; c + 64 <= bn; c += 64) {
-                uint8_t* sbuf = my_stage + (size_t)(out_flip & 1) * P_OUT_BUF_BYTES;
-                if (lane == 0) ptx::bulk_wait_group_read<1>();      // the store that used this buffer has read it
-                __syncwarp();
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t v[32];
-                    ptx::tmem_ld_32x32(taddr + (uint32_t)(c + 32 * h), v);
-                    ptx::tmem_ld_wait();
-                    const float* sc = tail->scale + c + 32 * h;
-                    const float* bi = tail->bias + c + 32 * h;
-#pragma unroll
-                    for (int j = 0; j < 32; j += 8) {
-                        uint32_t o[4];
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            float f0 = __fmul_rn(__int2float_rn((int)v[j + 2 * q]), out_scale(per_row, s_row, sc[j + 2 * q]));
-                            float f1 = __fmul_rn(__int2float_rn((int)v[j + 2 * q + 1]),
-                                                 out_scale(per_row, s_row, sc[j + 2 * q + 1]));
-                            if (has_bias) {
-                                f0 = __fadd_rn(f0, bi[j + 2 * q]);
-                                f1 = __fadd_rn(f1, bi[j + 2 * q + 1]);
-                            }
-                            o[q] = narrow2<BF>(f0, f1);
-                        }
-                        const int piece = 4 * h + (j >> 3);           // 16-byte piece of the 128-byte row
-                        *reinterpret_cast<uint4*>(sbuf + lane * 128 + ((piece ^ (lane & 7)) << 4)) =
-                            make_uint4(o[0], o[1], o[2], o[3]);
-                        if (arow != nullptr && row_ok && (n0 + c + 32 * h + j) < p.N) {
-                            int32_t* a = arow + c + 32 * h + j;
-                            *reinterpret_cast<uint4*>(a) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                            *reinterpret_cast<uint4*>(a + 4) = make_uint4(v[j + 4], v[j + 5], v[j + 6], v[j + 7]);
-                        }
-                    }
-                }
-                ptx::fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) {
-                    ptx::tma_store_2d_hint(tmap_y64, sbuf, n0 + c, row0, y_policy);
-                    ptx::bulk_commit_group();
-                }
-                ++out_flip;
-            }
-#pragma unroll 1
-            for (; c < bn; c += 16) {       // 16-column pieces: 32-byte rows, 32-byte swizzle
-                uint8_t* sbuf = my_stage + (size_t)(out_flip & 1) * P_OUT_BUF_BYTES;
-                if (lane == 0) ptx::bulk_wait_group_read<1>();
-                __syncwarp();
-                uint32_t v[16];
-                ptx::tmem_ld_32x16(taddr + (uint32_t)c, v);
-                ptx::tmem_ld_wait();
-                const float* sc = tail->scale + c;
-                const float* bi = tail->bias + c;
-#pragma unroll
-                for (int j = 0; j < 16; j += 8) {
-                    uint32_t o[4];
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        float f0 = __fmul_rn(__int2float_rn((int)v[j + 2 * q]), out_scale(per_row, s_row, sc[j + 2 * q]));
-                        float f1 = __fmul_rn(__int2float_rn((int)v[j + 2 * q + 1]),
-                                                 out_scale(per_row, s_row, sc[j + 2 * q + 1]));
-                        if (has_bias) {
-                            f0 = __fadd_rn(f0, bi[j + 2 * q]);
-                            f1 = __fadd_rn(f1, bi[j + 2 * q + 1]);
-                        }
-                        o[q] = narrow2<BF>(f0, f1);
-                    }
-                    const int piece = j >> 3;
-                    *reinterpret_cast<uint4*>(sbuf + lane * 32 + ((piece ^ ((lane >> 2) & 1)) << 4)) =
-                        make_uint4(o[0], o[1], o[2], o[3]);
-                    if (arow != nullptr && row_ok && (n0 + c + j) < p.N) {
-                        int32_t* a = arow + c + j;
-                        *reinterpret_cast<uint4*>(a) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                        *reinterpret_cast<uint4*>(a + 4) = make_uint4(v[j + 4], v[j + 5], v[j + 6], v[j + 7]);
-                    }
-                }
-                ptx::fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) {
-                    ptx::tma_store_2d_hint(tmap_y16, sbuf, n0 + c, row0, y_policy);
-                    ptx::bulk_commit_group();
-                }
-                ++out_flip;
-            }
-            // this warp has drained the accumulator buffer: tell the leader's MMA issuer
+            t.p = &p;
+            t.y64 = &maps.y64[q];
+            t.y16 = &maps.y16[q];
+            t.policy = y_policy;
+            t.taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * 256);
+            t.row0 = m_blk * PBM + (int)rank * 128 + quad * 32;
+            t.scale = tail->scale;
+            t.bias = tail->bias;
+            epilogue_units<BF>(t, my_stage, out_flip, lane, worker, last ? LAST_TILE_WORKERS : 1, last);
             ptx::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive_cluster(ptx::mapa_u32(ptx::smem_u32(&tail->tmem_empty[buf]), 0));
+            if (!helper && !last) {
+                // this warp has drained the accumulator buffer: tell the leader's MMA issuer (after the last tile
+                // nobody waits for it any more, and the arrival's release would wait for the copy-out stores)
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive_cluster(ptx::mapa_u32(ptx::smem_u32(&tail->tmem_empty[buf]), 0));
+            }
         }
+        // a pair that gave up before its last tile still has its quantizer warps waiting for the hand-over
+        if (!helper && any_tile && !helpers_released) asm volatile("bar.arrive 3, 384;" ::: "memory");
         // the output stores have read their shared-memory source; the writes themselves are complete by the end of
         // the grid, which is all that a later kernel or the host can observe
         if (lane == 0) ptx::bulk_wait_group_read<0>();
