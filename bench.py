@@ -183,6 +183,7 @@ class Stack:
 
     def __init__(self, P, device, rank: int, layers: int, tokens: int, training: bool = True):
         self.P, self.layers, self.tokens = P, layers, tokens
+        self.stream = torch.cuda.current_stream().cuda_stream      # raw handle: the cheapest thing to pass per call
         dt = torch.bfloat16
         self.x, self.g, self.y, self.dx, self.out = [], [], [], [], []
         self.w_int = [[None] * 7 for _ in range(layers)]
@@ -235,13 +236,14 @@ class Stack:
     # kernels launched per step: one fused quantizer launch per layer (the reduction's second stage runs in its
     # last block), then the linears (activation quantizer inside the GEMM kernel)
     def phase_a_layer(self, layer: int):
-        self.P.sasq_fakequant_fwd_bwd_multi(self.descs, self.scales[layer], self.grads[layer], self.q_ws, BITS)
+        self.P.sasq_fakequant_fwd_bwd_multi(self.descs, self.scales[layer], self.grads[layer], self.q_ws, BITS,
+                                            stream=self.stream)
         return 1
 
     def phase_b_layer(self, layer: int):
         n = 0
         for problems, launches in self.calls[layer]:
-            self.P.sasq_static_w8a8_linear_multi(problems, self.l_ws, bits=BITS)
+            self.P.sasq_static_w8a8_linear_multi(problems, self.l_ws, bits=BITS, stream=self.stream)
             n += launches
         return n
 
@@ -327,9 +329,11 @@ def quantizer_modes(P, stack, tokens: int, seconds: float):
     return out
 
 
-def linears_by_calls(P, stack, tokens: int, seconds: float, modes=("each", "dependent", "layer")):
+def linears_by_calls(P, stack, tokens: int, seconds: float, modes=("each", "dependent", "layer"), graph: bool = False):
     """The seven static linears of a layer at `tokens` rows, back to back, for each way of submitting them; the
-    layers' weights take turns so that no repetition finds its weights in L2."""
+    layers' weights take turns so that no repetition finds its weights in L2.  graph: the calls of up to eight
+    layers are captured once into a CUDA graph and the graph is replayed, which takes the host's per-call cost
+    (a few microseconds, more than a decode-sized kernel runs) out of the measurement; times are per layer."""
     ops = linear_ops(tokens)
     out = {}
     for name in modes:
@@ -339,10 +343,31 @@ def linears_by_calls(P, stack, tokens: int, seconds: float, modes=("each", "depe
 
         def run():
             for problems in tables[turn[0] % len(tables)]:
-                P.sasq_static_w8a8_linear_multi(problems, stack.l_ws, bits=BITS)
+                P.sasq_static_w8a8_linear_multi(problems, stack.l_ws, bits=BITS, stream=stack.stream)
             turn[0] += 1
 
-        ms = timed_reps(run, seconds)
+        per = 1
+        if graph:
+            per = min(8, len(tables))
+            for _ in range(per):
+                run()                           # one-time set-up of every shape happens outside the capture
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            handle = stack.stream
+            with torch.cuda.stream(side):
+                stack.stream = side.cuda_stream
+                turn[0] = 0
+                with torch.cuda.graph(g, stream=side):
+                    for _ in range(per):
+                        run()
+            stack.stream = handle
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            ms = [m / per for m in timed_reps(g.replay, seconds)]
+        else:
+            ms = timed_reps(run, seconds)
         med, mn = med_min(ms)
         out[name] = {"us_median": round(med * 1e3, 2), "us_min": round(mn * 1e3, 2),
                      "tops_median": round(ops / (med * 1e-3) / 1e12, 2), "tops_best": round(ops / (mn * 1e-3) / 1e12, 2),
@@ -463,6 +488,8 @@ def run_ours(args):
         for t3 in CONFIG3_TOKENS:
             if t3 <= T:
                 cfg3[f"T{t3}"] = linears_by_calls(P, stack, t3, 0.3 if t3 >= 2048 else 0.15)
+                if t3 <= 128:       # decode sizes: also with the host's per-call cost taken out
+                    cfg3[f"T{t3}_graph_replay"] = linears_by_calls(P, stack, t3, 0.15, graph=True)
         context["config3_one_layer_by_tokens"] = cfg3
         if T >= 2048:
             context["config2_quantizer_T2048"] = quantizer_modes(P, stack, 2048, 0.3)["fused"]

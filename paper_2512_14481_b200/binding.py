@@ -186,6 +186,9 @@ def _ptr(t) -> int | None:
 
 
 def _stream(stream) -> int:
+    """None: torch's current stream; a torch stream; or a raw cudaStream_t handle as an int (the cheapest to pass)."""
+    if isinstance(stream, int):
+        return stream
     s = torch.cuda.current_stream() if stream is None else stream
     return s.cuda_stream
 
@@ -499,15 +502,19 @@ class LinearProblems:
         self.descs, dt = _linear_descs(self.problems)
         self.dt = SASQ_BF16 if dt is None else dt
         self.count = len(self.problems)
+        self._ws = None         # (workspace tensor, pointer, bytes) of the last call: checked once per workspace
 
 
 def sasq_static_w8a8_linear_multi(problems, workspace, bits: int = 8, stream=None) -> None:
     """Independent static W8A8 linears submitted together: a sequence of tuples (see _linear_descs) or a
     LinearProblems made from one."""
     prepared = problems if isinstance(problems, LinearProblems) else LinearProblems(problems)
-    _dev(workspace, "workspace")
+    ws = prepared._ws
+    if ws is None or ws[0] is not workspace:
+        _dev(workspace, "workspace")
+        ws = prepared._ws = (workspace, _ptr(workspace), _nbytes(workspace))
     _check(load_library().sasq_static_w8a8_linear_multi(prepared.count, prepared.descs, prepared.dt, int(bits),
-                                                        _ptr(workspace), _nbytes(workspace), _stream(stream)),
+                                                        ws[1], ws[2], _stream(stream)),
            "sasq_static_w8a8_linear_multi")
 
 

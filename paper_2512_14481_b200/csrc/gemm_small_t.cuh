@@ -16,14 +16,24 @@ namespace {
 // (int32: exact in any order), dequantises and stores them.
 //   warp 0      TMA producer: W tile (128 x 128 B) + int8 activation tile (TP x 128 B) per stage
 //   warp 1      MMA issuer
-//   warps 2..5  first the activation quantizer (Eq. 1 with the fixed factor, all CTAs share the T x K elements and
-//               publish through one counter; the producers load activation tiles only after it is complete, the
-//               weight tiles of the first stages are on their way by then), then the epilogue
+//   warps 2..5  first the activation quantizer (Eq. 1 with the fixed factor), then the epilogue.  Up to 16 rows every
+//               CTA quantizes what its own K slice needs straight into the activation tiles of its stages: a row
+//               block this small is cheaper to convert 32 times over than to pass through global memory, a counter
+//               and a second set of loads (3 us of a 10 us launch, measured).  Above that all CTAs share the T x K
+//               elements and publish through one counter; the producers load activation tiles only after it is
+//               complete, the weight tiles of the first stages are on their way by then
 // ---------------------------------------------------------------------------
 constexpr int D_THREADS = 192;
 constexpr int D_W_BYTES = 128 * BK;          // weight tile of a stage
 constexpr int D_MAX_STAGES = 8;
 constexpr int D_RING_BYTES = 192 * 1024;     // stages x (weight tile + activation tile) fit in here
+// With T <= 16 a launch is one latency chain (set-up, weights, a few MMAs, reduction, stores) and nothing in it is
+// long enough to hide the others.  Such launches take a little less than half of an SM's shared memory, so that
+// the CTAs of the NEXT launch of the stream are resident beside them from the start and have their first weight
+// tiles in shared memory by the time the kernel before them has finished (the weights are frozen: they are
+// requested before the wait on the earlier kernel).
+constexpr int D_RING_BYTES_LITE = 108 * 1024;
+constexpr int D_LITE_MAX_TP = 16;        // (at 32 rows converting the rows in every CTA was measured slower: 134 against 113 us)
 
 struct DecodeTail {
     uint64_t full[D_MAX_STAGES];
@@ -55,8 +65,12 @@ struct DecodeParams {
     int split;           // CTAs per cluster = K slices
     int n_tiles;         // 128-channel tiles of all problems
     uint32_t tmem_cols;  // power of two >= max(32, tp)
+    int ring_bytes;      // D_RING_BYTES or D_RING_BYTES_LITE: stages and reduction slots; the barriers follow
     int slots_offset;    // byte offset of the reduction slots in the CTA's shared memory: behind the stages, never
                          // under them, because peers write there while this CTA may still be in its mainloop
+    bool local_x;        // T <= 16 with static factors: every CTA quantizes the part of x its own K slice needs
+                         // straight into the activation tiles of its pipeline stages (no codes in global memory, no
+                         // counter, no activation loads); `quantize`, `ready` and `done` are then unused
     bool quantize;       // the activation quantizer runs inside this launch
     unsigned* ready;     // [count] per problem: 16-element items quantized and visible; zero at launch
     unsigned* done;
@@ -84,12 +98,76 @@ __device__ __forceinline__ bool wait_bounded_d(uint64_t* bar, uint32_t parity, D
     return true;
 }
 
+// Eq. 1 with the fixed factor on the tp x 128 elements of every k-block of a CTA's K slice, written as int8 codes
+// into the activation tile of the k-block's pipeline stage: rows of 128 bytes with the 128-byte swizzle the MMA's
+// descriptor expects (16-byte piece c of row r sits at piece c ^ (r & 7)).  Run by the 128 threads of warps 2..5.
+// One item = 8 adjacent elements of a row (one 128-bit load); a k-block has tp x 16 items, PER per thread; rows >= T
+// and columns >= K are zeros.  The words of DEPTH k-blocks are in flight per thread: a slot is refilled as soon as
+// it has been converted, so the loads' latency is paid once, not once per k-block.
+template <bool BF, int PER, int DEPTH>
+__device__ __forceinline__ void local_activation_tiles(const DecodeParams& dp, const DecodeProblem& me, DecodeTail* tail,
+                                                       uint8_t* ring, int stage_bytes, int kb_begin, int kb_end, int et,
+                                                       int lane) {
+    const LinearParams& p = me.lp;
+    const bool one = p.chan_inv == nullptr;                       // one static factor for the whole tensor
+    const uint4* xsrc = reinterpret_cast<const uint4*>(me.x);
+    const int vec_per_row = p.K >> 3;
+    const int items_per_kb = dp.tp * 16;
+    uint4 buf[DEPTH][PER];
+    auto load_kb = [&](int kb, uint4 (&v)[PER]) {
+#pragma unroll
+        for (int u = 0; u < PER; ++u) {
+            const int item = et + 128 * u;
+            const int r = item >> 4, c8 = kb * 16 + (item & 15);                  // row, 8-element column group
+            v[u] = (item < items_per_kb && r < p.T && c8 < vec_per_row) ? ld_stream16(xsrc + (size_t)r * vec_per_row + c8)
+                                                                         : make_uint4(0u, 0u, 0u, 0u);
+        }
+    };
+#pragma unroll
+    for (int d = 0; d < DEPTH; ++d)
+        if (kb_begin + d < kb_end) load_kb(kb_begin + d, buf[d]);
+    // the factor is fetched with the first loads already in flight
+    const float sxq = one ? __ldg(p.x_scale) : 1.0f;
+    if (one && blockIdx.x == 0 && et == 0 && scale_is_bad(sxq)) atomicMax(p.status, (int)SASQ_ERR_BAD_SCALE);
+    const float inv = __fdiv_rn(1.0f, sxq);
+    int stage = 0;
+    uint32_t phase = 0;
+    for (int base = kb_begin; base < kb_end; base += DEPTH) {
+#pragma unroll
+        for (int d = 0; d < DEPTH; ++d) {
+            const int kb = base + d;
+            if (kb < kb_end) {
+                if (kb - kb_begin >= dp.stages) {           // the MMAs that read this tile before have completed
+                    if (!wait_bounded_d(&tail->empty[stage], phase ^ 1u, tail, p)) return;
+                }
+                uint8_t* x_tile = ring + (size_t)stage * stage_bytes + D_W_BYTES;
+#pragma unroll
+                for (int u = 0; u < PER; ++u) {
+                    const int item = et + 128 * u;
+                    if (item < items_per_kb) {
+                        const int r = item >> 4, j = item & 15;
+                        const uint2 codes = one ? quantize8<BF, false>(buf[d][u], inv, dp.qn, dp.qp)
+                                                : quantize8_channels<BF>(buf[d][u], p.chan_inv + 8 * (kb * 16 + j), dp.qn,
+                                                                         dp.qp);
+                        *reinterpret_cast<uint2*>(x_tile + r * 128 + (((j >> 1) ^ (r & 7)) << 4) + ((j & 1) << 3)) = codes;
+                    }
+                }
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&tail->full[stage]);
+                if (kb + DEPTH < kb_end) load_kb(kb + DEPTH, buf[d]);
+                if (++stage == dp.stages) { stage = 0; phase ^= 1u; }
+            }
+        }
+    }
+}
+
 template <bool BF>
 __global__ void __launch_bounds__(D_THREADS, 1)
 w8a8_decode_kernel(const __grid_constant__ DecodeMaps maps, const __grid_constant__ DecodeParams dp) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* ring = smem_raw;
-    DecodeTail* tail = reinterpret_cast<DecodeTail*>(ring + D_RING_BYTES);
+    DecodeTail* tail = reinterpret_cast<DecodeTail*>(ring + dp.ring_bytes);
     // the problem this cluster's tile belongs to
     const int tile_all = blockIdx.x / dp.split;
     int q_mine = 0;
@@ -116,14 +194,16 @@ w8a8_decode_kernel(const __grid_constant__ DecodeMaps maps, const __grid_constan
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < dp.stages; ++s) {
-            ptx::mbar_init(&tail->full[s], 1);
+            // a stage is full when its weight tile has landed (the producer's arrival with the byte count) and, with
+            // local activation tiles, when each of the four quantizer warps has written its share of the tile
+            ptx::mbar_init(&tail->full[s], dp.local_x ? 5 : 1);
             ptx::mbar_init(&tail->empty[s], 1);
         }
         ptx::mbar_init(&tail->acc_full, 1);
         tail->abort_flag = 0;
         ptx::mbar_init_fence();
         ptx::prefetch_tensormap(tmap_w);
-        ptx::prefetch_tensormap(tmap_x);
+        if (!dp.local_x) ptx::prefetch_tensormap(tmap_x);
     }
     if (warp == 1) {
         ptx::tmem_alloc(&tail->tmem_base, dp.tmem_cols);
@@ -133,10 +213,14 @@ w8a8_decode_kernel(const __grid_constant__ DecodeMaps maps, const __grid_constan
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = tail->tmem_base;
-    pdl_wait();                         // set-up done; from here on global memory of earlier kernels is used
+    // Set-up done.  From here on memory that earlier kernels of the stream may have written (x, the factors) or may
+    // still be using (y, the workspace) is touched; the producer warp first requests its weight tiles, which depend on
+    // no earlier kernel, and waits afterwards.
+    if (warp != 0) pdl_wait();
 
     // 16-element items the in-kernel quantizer has to publish (none if the activations came quantized)
-    const unsigned items_total = dp.quantize ? (unsigned)(((long long)p.T * p.K) >> 4) : 0u;   // of this CTA's problem
+    const unsigned items_total =
+        (dp.quantize && !dp.local_x) ? (unsigned)(((long long)p.T * p.K) >> 4) : 0u;             // of this CTA's problem
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
@@ -147,10 +231,12 @@ w8a8_decode_kernel(const __grid_constant__ DecodeMaps maps, const __grid_constan
             // weight tiles of the first stages go out at once; the activation tiles follow when every CTA has
             // quantized its share of x
             int early = kb_end - kb_begin < dp.stages ? kb_end - kb_begin : dp.stages;
+            const uint32_t stage_tx = dp.local_x ? (uint32_t)D_W_BYTES : (uint32_t)stage_bytes;
             for (int i = 0; i < early; ++i) {
-                ptx::mbar_arrive_expect_tx(&tail->full[i], (uint32_t)stage_bytes);
+                ptx::mbar_arrive_expect_tx(&tail->full[i], stage_tx);
                 ptx::tma_load_2d(ring + (size_t)i * stage_bytes, tmap_w, &tail->full[i], (kb_begin + i) * BK, n0);
             }
+            pdl_wait();
             if (items_total != 0) {
                 const long long t0 = clock64();
                 int polls = 0;
@@ -176,10 +262,10 @@ w8a8_decode_kernel(const __grid_constant__ DecodeMaps maps, const __grid_constan
                 if (kb - kb_begin >= early) {
                     ok = wait_bounded_d(&tail->empty[stage], phase ^ 1u, tail, p);
                     if (!ok) break;
-                    ptx::mbar_arrive_expect_tx(&tail->full[stage], (uint32_t)stage_bytes);
+                    ptx::mbar_arrive_expect_tx(&tail->full[stage], stage_tx);
                     ptx::tma_load_2d(w_dst, tmap_w, &tail->full[stage], kb * BK, n0);
                 }
-                ptx::tma_load_2d(w_dst + D_W_BYTES, tmap_x, &tail->full[stage], kb * BK, 0);
+                if (!dp.local_x) ptx::tma_load_2d(w_dst + D_W_BYTES, tmap_x, &tail->full[stage], kb * BK, 0);
                 if (++stage == dp.stages) { stage = 0; phase ^= 1u; }
             }
             if (!ok) {      // copies in flight must land before the CTA's shared memory goes away
@@ -219,7 +305,10 @@ w8a8_decode_kernel(const __grid_constant__ DecodeMaps maps, const __grid_constan
     } else {
         // ---------------- activation quantizer, then epilogue (warps 2..5) ----------------
         const int et = threadIdx.x - 64;                       // 0..127
-        if (dp.quantize && dp.row_scale_out != nullptr) {
+        if (dp.local_x) {
+            local_activation_tiles<BF, (D_LITE_MAX_TP * 16) / 128, 8>(dp, me, tail, ring, stage_bytes, kb_begin, kb_end, et,
+                                                                      lane);
+        } else if (dp.quantize && dp.row_scale_out != nullptr) {
             // Dynamic per-token quantization (Sec. 4.4, generation phase) inside the launch: the rows are dealt to
             // the CTAs, and the 128 quantizer threads of a CTA take a row together.  The row's factor is its own
             // max-based one, s_t = max_k |x[t,k]| / Qp (Eq. 1; an all-zero row takes s_t = 1).  Each thread keeps its
@@ -355,6 +444,17 @@ w8a8_decode_kernel(const __grid_constant__ DecodeMaps maps, const __grid_constan
     // a role gave up after a bounded wait and the status word says so; the sums below are then garbage but every
     // access stays in bounds).  Nobody touches another CTA's shared memory afterwards, so the CTAs may finish
     // independently.
+    // what the stores below need from global memory is requested before the barrier, not after it
+    float pre_sx = 1.0f, pre_ws = 0.0f, pre_bias = 0.0f;
+    if (warp >= 2) {
+        const int rows_own = 128 / dp.split;
+        const int n_first = n0 + rank * rows_own + (threadIdx.x - 64) % rows_own;
+        if (p.row_scale == nullptr && p.chan_inv == nullptr) pre_sx = __ldg(p.x_scale);
+        if (n_first < p.N) {
+            pre_ws = __ldg(p.w_scale + n_first);
+            if (p.bias != nullptr) pre_bias = widen1<BF>(__ldg(reinterpret_cast<const uint16_t*>(p.bias) + n_first));
+        }
+    }
     __syncthreads();
     ptx::cluster_sync_all();
 
@@ -367,7 +467,7 @@ w8a8_decode_kernel(const __grid_constant__ DecodeMaps maps, const __grid_constan
         const int pstride = dp.tp + 4;
         const bool has_bias = p.bias != nullptr;
         const bool per_row = p.row_scale != nullptr;
-        const float sx = (per_row || p.chan_inv != nullptr) ? 1.0f : __ldg(p.x_scale);
+        const float sx = pre_sx;
         const int items = rows * (dp.tp >> 2);
         const int32_t* slots = reinterpret_cast<const int32_t*>(ring + dp.slots_offset);
         for (int it = et; it < items; it += 128) {
@@ -380,9 +480,12 @@ w8a8_decode_kernel(const __grid_constant__ DecodeMaps maps, const __grid_constan
                 acc[0] += v.x; acc[1] += v.y; acc[2] += v.z; acc[3] += v.w;
             }
             if (n < p.N) {
-                const float ws = __ldg(p.w_scale + n);
+                const bool first = it == et;            // this thread's first item: its factors are here already
+                const float ws = first ? pre_ws : __ldg(p.w_scale + n);
                 const float sc = __fmul_rn(sx, ws);
-                const float bv = has_bias ? widen1<BF>(__ldg(reinterpret_cast<const uint16_t*>(p.bias) + n)) : 0.0f;
+                const float bv = !has_bias ? 0.0f
+                                 : first   ? pre_bias
+                                           : widen1<BF>(__ldg(reinterpret_cast<const uint16_t*>(p.bias) + n));
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const int t = t0 + j;
@@ -407,7 +510,7 @@ w8a8_decode_kernel(const __grid_constant__ DecodeMaps maps, const __grid_constan
         ptx::tmem_dealloc(tmem_base, dp.tmem_cols);
     }
     // the CTA that finishes last leaves the counters at zero for the next launch that draws them
-    if (dp.quantize && threadIdx.x == 0) {
+    if (dp.quantize && !dp.local_x && threadIdx.x == 0) {
         if (atomicAdd(dp.done, 1u) == gridDim.x - 1) {
             for (int q = 0; q < dp.count; ++q) dp.ready[q] = 0u;
             *dp.done = 0u;

@@ -225,28 +225,37 @@ int pair_capacity(bool bf, int sm_count) {
     return clusters;
 }
 
+// Shared memory of a small-T launch with T rows: the smaller footprint (two CTAs per SM) up to D_LITE_MAX_TP rows.
+int decode_ring_bytes(int64_t T) {
+    const int64_t tp = (T + 15) / 16 * 16;
+    return tp <= D_LITE_MAX_TP ? D_RING_BYTES_LITE : D_RING_BYTES;
+}
+
 // Largest K split (CTAs per cluster) of the small-T kernel with which all n_tiles clusters are resident at once (the
-// in-kernel activation quantizer needs every CTA of the grid running); 0 if even one CTA per tile does not fit.
-int decode_split(bool bf, int n_tiles, int k_blocks, int sm_count, size_t smem_bytes) {
+// in-kernel activation quantizer needs every CTA of the grid running) on at most one CTA per SM (with the smaller
+// footprint the other half of each SM is left to the launch that follows); 0 if even one CTA per tile does not fit.
+int decode_split(bool bf, int n_tiles, int k_blocks, int sm_count, int ring_bytes) {
     static int ready[64][2] = {};
-    static int cap[64][2][4] = {};            // resident clusters for S = 1, 2, 4, 8; 0 = not asked yet
+    static int cap[64][2][2][4] = {};            // resident clusters for S = 1, 2, 4, 8; 0 = not asked yet
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
     const void* fn = bf ? reinterpret_cast<const void*>(w8a8_decode_kernel<true>)
                         : reinterpret_cast<const void*>(w8a8_decode_kernel<false>);
     if (!ready[dev][bf]) {
-        if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)(D_RING_BYTES + sizeof(DecodeTail))) != cudaSuccess)
             return 0;
         ready[dev][bf] = 1;
     }
+    const int lite = ring_bytes == D_RING_BYTES_LITE ? 1 : 0;
     for (int si = 3; si >= 0; --si) {
         const int S = 1 << si;
         if (S > k_blocks || (long long)n_tiles * S > sm_count) continue;
-        if (cap[dev][bf][si] == 0) {
+        if (cap[dev][bf][lite][si] == 0) {
             cudaLaunchConfig_t cfg{};
             cfg.gridDim = dim3((unsigned)(sm_count / S * S), 1, 1);
             cfg.blockDim = dim3(D_THREADS, 1, 1);
-            cfg.dynamicSmemBytes = smem_bytes;
+            cfg.dynamicSmemBytes = (size_t)ring_bytes + sizeof(DecodeTail);
             cudaLaunchAttribute attr[1];
             attr[0].id = cudaLaunchAttributeClusterDimension;
             attr[0].val.clusterDim.x = (unsigned)S;
@@ -256,9 +265,9 @@ int decode_split(bool bf, int n_tiles, int k_blocks, int sm_count, size_t smem_b
             cfg.numAttrs = 1;
             int clusters = 0;
             if (cudaOccupancyMaxActiveClusters(&clusters, fn, &cfg) != cudaSuccess || clusters <= 0) clusters = -1;
-            cap[dev][bf][si] = clusters;
+            cap[dev][bf][lite][si] = clusters;
         }
-        if (cap[dev][bf][si] >= n_tiles) return S;
+        if (cap[dev][bf][lite][si] >= n_tiles) return S;
     }
     return 0;
 }
@@ -268,6 +277,23 @@ int decode_split(bool bf, int n_tiles, int k_blocks, int sm_count, size_t smem_b
 // launch takes as long as its fullest pair: waves x that cost of the widest tile.  Tiles are at least 16 x 8 = 128
 // columns wide unless N itself is narrower.  Fewer, wider tiles win ties (less fixed work per tile).
 void plan_pair_tiles(PairParams* pp, int m_blocks, long long N, int pairs) {
+    // the search below runs over up to N / 16 candidates; decode-sized calls are bound by the host, and a model has
+    // a handful of distinct shapes: the last few plans are kept per thread
+    struct Plan { int m_blocks, pairs; long long N; int n_tiles, base_units, rem_units, w_box_rows; };
+    constexpr int kPlans = 16;
+    thread_local Plan plans[kPlans] = {};
+    thread_local int next_plan = 0;
+    for (int i = 0; i < kPlans; ++i) {
+        const Plan& c = plans[i];
+        if (c.N == N && c.m_blocks == m_blocks && c.pairs == pairs && c.n_tiles != 0) {
+            pp->pair_m_blocks = m_blocks;
+            pp->n_tiles = c.n_tiles;
+            pp->base_units = c.base_units;
+            pp->rem_units = c.rem_units;
+            pp->w_box_rows = c.w_box_rows;
+            return;
+        }
+    }
     const int units = (int)((N + 15) / 16);
     int best_nt = (units + 15) / 16;
     double best_cost = -1.0;
@@ -285,6 +311,8 @@ void plan_pair_tiles(PairParams* pp, int m_blocks, long long N, int pairs) {
     pp->base_units = units / best_nt;
     pp->rem_units = units % best_nt;
     pp->w_box_rows = 8 * (pp->base_units + (pp->rem_units ? 1 : 0));
+    plans[next_plan] = Plan{m_blocks, pairs, N, pp->n_tiles, pp->base_units, pp->rem_units, pp->w_box_rows};
+    next_plan = (next_plan + 1) % kPlans;
 }
 
 int* status_word_ptr() {
@@ -474,26 +502,30 @@ int launch_pair_group(const GroupMaps& maps, const GroupParams& gp, int pairs, b
 // n_tiles, quantize, qn, qp, row_scale_out and maps.w filled in by the caller): sets the shared geometry, draws the
 // counters, encodes the activation maps and launches n_tiles clusters of `split` CTAs.
 int launch_decode_group(DecodeMaps& maps, DecodeParams& dp, int T, int split, bool bf, cudaStream_t st) {
-    constexpr size_t kDecodeSmem = (size_t)D_RING_BYTES + sizeof(DecodeTail);
+    dp.ring_bytes = decode_ring_bytes(T);
+    const size_t smem_bytes = (size_t)dp.ring_bytes + sizeof(DecodeTail);
     dp.tp = (T + 15) / 16 * 16;
     const int stage_bytes = D_W_BYTES + dp.tp * BK;
     const int slot_bytes = (128 * (dp.tp + 4) * 4 + 1023) & ~1023;          // S x (128 / S) rows of tp + 4 words
-    const int ring_bytes = D_RING_BYTES - slot_bytes;
+    const int ring_bytes = dp.ring_bytes - slot_bytes;
     dp.slots_offset = ring_bytes;
     dp.stages = ring_bytes / stage_bytes < D_MAX_STAGES ? ring_bytes / stage_bytes : D_MAX_STAGES;
     dp.split = split;
     dp.tmem_cols = 32;
     while ((int)dp.tmem_cols < dp.tp) dp.tmem_cols <<= 1;
-    if (dp.quantize) {
+    // static factors and at most 16 rows: the CTAs quantize their own activation tiles in shared memory
+    dp.local_x = dp.quantize && dp.row_scale_out == nullptr && dp.tp <= D_LITE_MAX_TP;
+    if (dp.quantize && !dp.local_x) {
         const int rc = next_ready_slot(st, dp.count, &dp.ready, &dp.done);
         if (rc != SASQ_OK) return rc;
     }
-    for (int q = 0; q < dp.count; ++q)
-        if (!make_tmap(&maps.x[q], dp.prob[q].a_int8, T, dp.prob[q].lp.K, dp.tp)) return SASQ_ERR_CUDA;
+    if (!dp.local_x)
+        for (int q = 0; q < dp.count; ++q)
+            if (!make_tmap(&maps.x[q], dp.prob[q].a_int8, T, dp.prob[q].lp.K, dp.tp)) return SASQ_ERR_CUDA;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)(dp.n_tiles * split), 1, 1);
     cfg.blockDim = dim3(D_THREADS, 1, 1);
-    cfg.dynamicSmemBytes = kDecodeSmem;
+    cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[3];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -504,7 +536,8 @@ int launch_decode_group(DecodeMaps& maps, DecodeParams& dp, int T, int split, bo
     attr[2].id = cudaLaunchAttributeCooperative;
     attr[2].val.cooperative = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = (dp.quantize && g_gang_launch.load(std::memory_order_relaxed)) ? 3 : 2;
+    // with local activation tiles no CTA waits for another launch-mate outside its own cluster
+    cfg.numAttrs = (dp.quantize && !dp.local_x && g_gang_launch.load(std::memory_order_relaxed)) ? 3 : 2;
     cudaError_t e;
     if (bf) e = cudaLaunchKernelEx(&cfg, w8a8_decode_kernel<true>, maps, dp);
     else e = cudaLaunchKernelEx(&cfg, w8a8_decode_kernel<false>, maps, dp);
@@ -615,10 +648,9 @@ int linear_impl(const void* x, const int8_t* w, const float* w_scale, const floa
     uint8_t* a_int8 = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(workspace) + 127) & ~uintptr_t(127));
     const float qn = (float)(1 << (bits - 1)), qp = (float)((1 << (bits - 1)) - 1);
     const int k_blocks = (int)((K + BK - 1) / BK);
-    constexpr size_t kDecodeSmem = (size_t)D_RING_BYTES + sizeof(DecodeTail);
     const int n_tiles128 = (int)((N + 127) / 128);
     const int split = (T <= BM && n_tiles128 <= sm_count)
-                          ? decode_split(dt == SASQ_BF16, n_tiles128, k_blocks, sm_count, kDecodeSmem) : 0;
+                          ? decode_split(dt == SASQ_BF16, n_tiles128, k_blocks, sm_count, decode_ring_bytes(T)) : 0;
     const bool in_kernel_quantizer = !dynamic && (split > 0 || (T > BM && (T + PBM - 1) / PBM <= kMaxRowBlocks));
     const float* row_scale = nullptr;
     const float* chan_inv = nullptr;
@@ -908,8 +940,7 @@ int sasq_static_w8a8_linear_multi(int count, const sasq_linear_desc_t* descs_hos
         dp.quantize = true;
         dp.qn = qn;
         dp.qp = qp;
-        constexpr size_t kDecodeSmem = (size_t)D_RING_BYTES + sizeof(DecodeTail);
-        const int split = decode_split(bf, dp.n_tiles, min_kblocks, sm_count, kDecodeSmem);
+        const int split = decode_split(bf, dp.n_tiles, min_kblocks, sm_count, decode_ring_bytes(T));
         if (split <= 0) {                        // cannot all be resident after all: one by one
             int rc = SASQ_OK;
             for (int i = first; i < last && rc == SASQ_OK; ++i)
