@@ -54,10 +54,10 @@ CPU_SAMPLE_TOKENS = 2048              # the oracle legs run on the first tokens 
 # DRAM bytes (read + write) per launch, from ncu captures of these kernels (dram__bytes_read.sum + dram__bytes_write.sum);
 # None whenever the kernel has changed since its capture.  Keyed by (kernel, tokens): traffic grows with the tokens.
 NCU_TRAFFIC = {
-    ("fakequant", 2048): None,
+    ("fakequant", 2048): 531.6e6,
     ("gemm_layer", 2048): None,
-    ("fakequant", 16384): None,
-    ("gemm_q_proj", 16384): None,
+    ("fakequant", 16384): 4617.0e6,
+    ("gemm_q_proj", 16384): 355.0e6,       # one q_proj launch, 16384 x 4096 x 4096 (285 MB algorithmic)
 }
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -275,13 +275,23 @@ def tensor_peak_for(region_s: float, peaks: dict, peak_kind: str):
     return peaks["bf16_tflops"] * INT8_OVER_BF16_NOMINAL, f"{peak_kind} burst bf16 x 2"
 
 
-def timed_reps(fn, min_seconds: float, min_reps: int = 5, max_reps: int = 2000):
-    """Runs fn() repeatedly, each repetition between its own pair of CUDA events, until `min_seconds` of device time
-    and `min_reps` repetitions have accumulated; returns the per-repetition milliseconds."""
+def timed_reps(fn, min_seconds: float, min_reps: int = 5, max_reps: int = 2000, back_to_back: int = 0):
+    """Runs fn() repeatedly between pairs of CUDA events until `min_seconds` of device time and `min_reps` samples
+    have accumulated; returns milliseconds per call.  A sample is `back_to_back` calls submitted one after the other
+    between one pair of events (0: as many as make a sample about a millisecond long, at most 50), so that short
+    kernels are timed the way they run in a step, each behind the one before, not each behind an idle device."""
     stream = torch.cuda.current_stream()
     for _ in range(3):
         fn()
     torch.cuda.synchronize()
+    inner = back_to_back
+    if inner <= 0:
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        fn()
+        b.record(stream)
+        torch.cuda.synchronize()
+        inner = int(max(1, min(50, round(1.0 / max(a.elapsed_time(b), 1e-3)))))
     out = []
     total = 0.0
     while (total < min_seconds * 1e3 or len(out) < min_reps) and len(out) < max_reps:
@@ -289,11 +299,12 @@ def timed_reps(fn, min_seconds: float, min_reps: int = 5, max_reps: int = 2000):
         ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(batch)]
         for a, b in ev:
             a.record(stream)
-            fn()
+            for _ in range(inner):
+                fn()
             b.record(stream)
         torch.cuda.synchronize()
         ms = [a.elapsed_time(b) for a, b in ev]
-        out += ms
+        out += [m / inner for m in ms]
         total += sum(ms)
     return out
 
@@ -372,6 +383,43 @@ def linears_by_calls(P, stack, tokens: int, seconds: float, modes=("each", "depe
         out[name] = {"us_median": round(med * 1e3, 2), "us_min": round(mn * 1e3, 2),
                      "tops_median": round(ops / (med * 1e-3) / 1e12, 2), "tops_best": round(ops / (mn * 1e-3) / 1e12, 2),
                      "weight_gbs_median": round(weight_bytes() / (med * 1e-3) / 1e9, 1), "reps": len(ms)}
+    return out
+
+
+def dynamic_per_token(P, stack, tokens: int, seconds: float):
+    """Sec. 4.4, generation phase: the seven linears of a layer with dynamic per-token factors at `tokens` rows, one
+    call per linear, submitted directly and replayed from a CUDA graph (times per layer)."""
+    ws = torch.empty(max(P.sasq_dynamic_w8a8_linear_workspace(tokens, N, K) for _, K, N in LINEARS), dtype=torch.uint8,
+                     device=stack.x[0].device)
+    turn = [0]
+    handle = [stack.stream]
+
+    def run():
+        layer = turn[0] % stack.layers
+        for i in range(7):
+            P.sasq_dynamic_w8a8_linear(stack.x[i][:tokens], stack.w_int[layer][i], stack.w_scale[layer][i],
+                                       stack.out[i][:tokens], workspace=ws, stream=handle[0])
+        turn[0] += 1
+
+    out = {}
+    ms = timed_reps(run, seconds)
+    out["direct"] = {"us_median": round(statistics.median(ms) * 1e3, 2), "us_min": round(min(ms) * 1e3, 2)}
+    per = min(8, stack.layers)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        handle[0] = side.cuda_stream
+        turn[0] = 0
+        with torch.cuda.graph(g, stream=side):
+            for _ in range(per):
+                run()
+    handle[0] = stack.stream
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    ms = [m / per for m in timed_reps(g.replay, seconds)]
+    out["graph_replay"] = {"us_median": round(statistics.median(ms) * 1e3, 2), "us_min": round(min(ms) * 1e3, 2)}
     return out
 
 
@@ -491,6 +539,7 @@ def run_ours(args):
                 if t3 <= 128:       # decode sizes: also with the host's per-call cost taken out
                     cfg3[f"T{t3}_graph_replay"] = linears_by_calls(P, stack, t3, 0.15, graph=True)
         context["config3_one_layer_by_tokens"] = cfg3
+        context["dynamic_per_token_T1"] = dynamic_per_token(P, stack, 1, 0.15)
         if T >= 2048:
             context["config2_quantizer_T2048"] = quantizer_modes(P, stack, 2048, 0.3)["fused"]
             P.sasq_set_gang_launch(True)          # what callers that overlap linears on several streams switch on
