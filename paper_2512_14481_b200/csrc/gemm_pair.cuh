@@ -27,17 +27,17 @@ namespace {
 // ---------------------------------------------------------------------------
 constexpr int PBM = 256;                 // rows per pair tile
 #ifndef SASQ_PAIR_STAGES
-#define SASQ_PAIR_STAGES 5
+#define SASQ_PAIR_STAGES 6       // 6 x 32 KB + 32 KB of output staging + barriers = 226 KB of the 227 KB a CTA may have
 #endif
 constexpr int P_STAGES = SASQ_PAIR_STAGES;
 constexpr int P_A_BYTES = 128 * BK;      // per CTA: 128 rows of A
 constexpr int P_B_BYTES_MAX = 128 * BK;  // per CTA: up to 128 rows of W
 constexpr int P_STAGE_BYTES = P_A_BYTES + P_B_BYTES_MAX;
 // A stage holds the CTA's half of the W tile first, then its rows of A.  The kernel exists in two layouts of the
-// same ring: 5 stages with all 128 rows of A, and, for launches whose problems all have T <= 32, 8 stages with 32
+// same ring: 6 stages with all 128 rows of A, and, for launches whose problems all have T <= 32, 9 stages with 32
 // rows of A (only the leader CTA has rows below T and loads them; the MMA still reads 128 rows from each CTA's
 // shared memory, the rest being whatever lies behind, and the accumulator rows they produce are never stored).
-// Such launches stream the weights once and are bound by the weight bytes in flight: 8 x 15 KB instead of 5 x 15 KB
+// Such launches stream the weights once and are bound by the weight bytes in flight: 9 x 15 KB instead of 6 x 15 KB
 // per CTA.
 constexpr int P_SMALL_ROWS = 32;
 constexpr int P_SMALL_STAGES = (P_STAGES * P_STAGE_BYTES) / (P_B_BYTES_MAX + P_SMALL_ROWS * BK);
@@ -57,6 +57,9 @@ constexpr int CONV_ITEMS = SASQ_CONV_ITEMS;
 constexpr int CONV_CHUNK = 32 * CONV_ITEMS;   // items per chunk (one warp)
 // The four epilogue warps of a CTA have nothing to drain until the first tile's accumulators are complete: they take
 // part in the first rounds of the chunk list as workers 8..11 of their CTA.
+#ifndef SASQ_PAIR_LOOK_AHEAD
+#define SASQ_PAIR_LOOK_AHEAD 1
+#endif
 #ifndef SASQ_EPI_CONV_ROUNDS
 #define SASQ_EPI_CONV_ROUNDS 1
 #endif
@@ -674,7 +677,34 @@ w8a8_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
                     ready_q = q;
                 }
                 if (!dep_waited) { pdl_wait(); dep_waited = true; }       // codes written by an earlier launch
+                // The check above costs a round trip to L2 and a proxy fence, and at the top of a tile the MMAs are
+                // about to run out of stages: once the ring is full of this tile's loads the producer looks ahead
+                // and, if the NEXT tile's row block is complete already (one load, no waiting), settles it here.
+                const int look_kb = p.k_blocks - 1 < STAGES ? p.k_blocks - 1 : STAGES;
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
+#if SASQ_PAIR_LOOK_AHEAD
+                    if (kb == look_kb) {
+                        TileWalk nw = walk;
+                        nw.next();
+                        if (nw.more()) {
+                            const int ng = nw.tile(gp);
+                            const int nq = problem_of(gp, ng);
+                            const PairParams& np = gp.prob[nq];
+                            const int n_blk = (ng - np.tile_begin) / np.n_tiles;
+                            if (np.x != nullptr && (n_blk != ready_blk || nq != ready_q)) {
+                                const int rows = np.lp.T - n_blk * PBM;
+                                const unsigned need = (unsigned)((rows < PBM ? rows : PBM) * (np.lp.K >> 3));
+                                unsigned v;
+                                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(np.ready + n_blk) : "memory");
+                                if (v >= need) {
+                                    asm volatile("fence.proxy.async.global;" ::: "memory");
+                                    ready_blk = n_blk;
+                                    ready_q = nq;
+                                }
+                            }
+                        }
+                    }
+#endif
                     uint8_t* w_dst = tiles + (size_t)stage * STAGE_BYTES;
                     // Only the leader arms the barrier (with the bytes of both CTAs); the partner's copies
                     // may complete first, which merely drives the transaction count negative for a while:
