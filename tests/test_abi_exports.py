@@ -77,6 +77,17 @@ def test_host_side_argument_errors_launch_nothing():
     assert lib.sasq_fakequant_fwd_bwd_multi(d, 2, a, a, 2, 0, 1, 8, a, 1 << 20, None) == INVALID
 
 
+def test_issue_rate_probe_rejects_bad_arguments_before_touching_a_device():
+    lib = P.load_library()
+    lib.sasq_debug_int8_issue_rate.restype = ctypes.c_int
+    lib.sasq_debug_int8_issue_rate.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_double),
+                                               ctypes.POINTER(ctypes.c_double), ctypes.c_void_p]
+    a, b = ctypes.c_double(0), ctypes.c_double(0)
+    assert lib.sasq_debug_int8_issue_rate(8, 256, ctypes.byref(a), ctypes.byref(b), None) == 1       # too few
+    assert lib.sasq_debug_int8_issue_rate(64, 260, ctypes.byref(a), ctypes.byref(b), None) == 1      # width
+    assert lib.sasq_debug_int8_issue_rate(64, 256, None, ctypes.byref(b), None) == 1                 # NULL output
+
+
 def test_binding_rejects_cpu_tensors():
     import torch
     x = torch.zeros(8, dtype=torch.bfloat16)

@@ -172,3 +172,16 @@ def test_unsupported_shapes_and_bad_scale_are_reported():
     P.sasq_static_w8a8_linear(x, w, ws, sc, y, workspace=wsp)
     assert P.sasq_device_status() == 4
     assert P.sasq_device_status() == 0
+
+
+@pytest.mark.parametrize("tag", [oracle.F16, oracle.BF16])
+@pytest.mark.parametrize("T,N,K,bits", [(1, 136, 144, 8), (5, 264, 1040, 8), (16, 520, 400, 8), (9, 4096, 11008, 8),
+                                        (16, 1032, 2064, 4), (3, 11008, 4096, 8), (17, 264, 1040, 8), (32, 520, 400, 8)])
+def test_parity_decode_sizes_with_ragged_k_and_bias(tag, T, N, K, bits):
+    """Up to 16 rows every CTA of the small-T kernel quantizes its own K slice into shared memory (K not a multiple of
+    128, rows padded to 16, slices of unequal length); 17 and 32 rows take the path through global memory.  All rows
+    and all accumulators against the oracle, with a bias and with a negative factor."""
+    xb, w_int, w_scale, s = make_case(T, N, K, tag, 7300 + T + N, bits=bits)
+    bias = oracle.bits_of((torch.randn(N, generator=torch.Generator().manual_seed(T)) * 0.5).to(DT[tag]))[0]
+    check(xb, tag, w_int, w_scale, s, bits=bits)
+    check(xb, tag, w_int, w_scale, -s, bits=bits, bias_bits=bias)
