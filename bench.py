@@ -55,9 +55,9 @@ CPU_SAMPLE_TOKENS = 2048              # the oracle legs run on the first tokens 
 # None whenever the kernel has changed since its capture.  Keyed by (kernel, tokens): traffic grows with the tokens.
 NCU_TRAFFIC = {
     ("fakequant", 2048): 531.6e6,
-    ("gemm_layer", 2048): None,
+    ("gemm_layer", 2048): 672.0e6,         # the seven linears of a layer in one launch (522 MB algorithmic)
     ("fakequant", 16384): 4617.0e6,
-    ("gemm_q_proj", 16384): 355.0e6,       # one q_proj launch, 16384 x 4096 x 4096 (285 MB algorithmic)
+    ("gemm_q_proj", 16384): 351.0e6,       # one q_proj launch, 16384 x 4096 x 4096 (285 MB algorithmic)
 }
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
