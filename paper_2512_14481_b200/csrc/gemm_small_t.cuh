@@ -422,7 +422,18 @@ w8a8_decode_kernel(const __grid_constant__ DecodeMaps maps, const __grid_constan
             const uint32_t dst = ptx::mapa_u32(local, (uint32_t)owner);
             if (kb_end > kb_begin) {
                 const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
-                for (int c = 0; c < dp.tp; c += 16) {
+                // 32 columns per read where the width allows: a read takes a few hundred cycles to come back
+                int c = 0;
+                for (; c + 32 <= dp.tp; c += 32) {
+                    uint32_t v[32];
+                    ptx::tmem_ld_32x32(taddr + (uint32_t)c, v);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (uint32_t)(c + 4 * j) * 4u),
+                                     "r"(v[4 * j]), "r"(v[4 * j + 1]), "r"(v[4 * j + 2]), "r"(v[4 * j + 3]) : "memory");
+                }
+                for (; c < dp.tp; c += 16) {
                     uint32_t v[16];
                     ptx::tmem_ld_32x16(taddr + (uint32_t)c, v);
                     ptx::tmem_ld_wait();
@@ -469,35 +480,79 @@ w8a8_decode_kernel(const __grid_constant__ DecodeMaps maps, const __grid_constan
         const bool per_row = p.row_scale != nullptr;
         const float sx = pre_sx;
         const int items = rows * (dp.tp >> 2);
-        const int32_t* slots = reinterpret_cast<const int32_t*>(ring + dp.slots_offset);
-        for (int it = et; it < items; it += 128) {
-            const int r_local = it % rows;
-            const int t0 = (it / rows) << 2;
-            const int n = n0 + rank * rows + r_local;
-            int32_t acc[4] = {0, 0, 0, 0};
-            for (int r = 0; r < dp.split; ++r) {
-                const int4 v = *reinterpret_cast<const int4*>(slots + (size_t)(r * rows + r_local) * pstride + t0);
-                acc[0] += v.x; acc[1] += v.y; acc[2] += v.z; acc[3] += v.w;
-            }
-            if (n < p.N) {
-                const bool first = it == et;            // this thread's first item: its factors are here already
-                const float ws = first ? pre_ws : __ldg(p.w_scale + n);
-                const float sc = __fmul_rn(sx, ws);
-                const float bv = !has_bias ? 0.0f
-                                 : first   ? pre_bias
-                                           : widen1<BF>(__ldg(reinterpret_cast<const uint16_t*>(p.bias) + n));
+        // rows divides 128, so a thread's items all belong to ONE channel: its factors were fetched before the
+        // barrier and are not loaded again per item (a dependent global load per item made this loop, not the
+        // weights, the longest part of a 128-row launch)
+        const int r_local = et % rows;
+        const int n = n0 + rank * rows + r_local;
+        const float ws = pre_ws;
+        const float sc = __fmul_rn(sx, ws);
+        const float bv = pre_bias;
+        // Four items at a time: first all their slot reads (explicit shared-memory loads: through generic pointers the
+        // compiler would have to keep every read behind the global stores before it), then their outputs, so that
+        // the latencies of the conversions and of the address arithmetic overlap instead of adding up (a thread has
+        // up to 32 items and a warp has the SM sub-partition to itself).
+        const int rows_log2 = 31 - __clz(rows);                 // rows is a power of two
+        const uint32_t slots_s = ptx::smem_u32(ring) + (uint32_t)dp.slots_offset;
+        // The outputs of the CTA (T tokens x rows channels) are gathered in shared memory, [token][channel], and then
+        // written with 128-bit stores: 2-byte stores, one channel per lane and one token per instruction, were the
+        // longest phase of a 128-row launch (13 us of 33 for 128 channels).  The pipeline stages are free by now:
+        // the accumulators this warp read were complete, so every load had landed and every MMA had read it.
+        uint16_t* y_stage = reinterpret_cast<uint16_t*>(ring);
+        int32_t* acc_n = p.acc_out != nullptr ? p.acc_out + n : nullptr;
+        const int T = p.T;
+        const size_t N = (size_t)p.N;
+        for (int it0 = et; it0 < items; it0 += 4 * 128) {
+            int32_t acc[4][4];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int t = t0 + j;
-                    if (t < p.T) {
-                        // a plain load: in the dynamic mode other CTAs wrote the factors during this launch
-                        const float sct = per_row ? __fmul_rn(p.row_scale[t], ws) : sc;
-                        float f = __fmul_rn(__int2float_rn(acc[j]), sct);
-                        if (has_bias) f = __fadd_rn(f, bv);
-                        reinterpret_cast<uint16_t*>(p.y)[(size_t)t * p.N + n] = narrow1<BF>(f);
-                        if (p.acc_out != nullptr) p.acc_out[(size_t)t * p.N + n] = acc[j];
+            for (int u = 0; u < 4; ++u) {
+                const int it = it0 + 128 * u;
+                acc[u][0] = acc[u][1] = acc[u][2] = acc[u][3] = 0;
+                if (it < items) {
+                    const int t0 = (it >> rows_log2) << 2;
+                    for (int r = 0; r < dp.split; ++r) {
+                        int4 v;
+                        asm volatile("ld.shared.v4.s32 {%0, %1, %2, %3}, [%4];"
+                                     : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                                     : "r"(slots_s + (uint32_t)(((r << rows_log2) + r_local) * pstride + t0) * 4u));
+                        acc[u][0] += v.x; acc[u][1] += v.y; acc[u][2] += v.z; acc[u][3] += v.w;
                     }
                 }
+            }
+            if (n < p.N) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int it = it0 + 128 * u;
+                    if (it < items) {
+                        const int t0 = (it >> rows_log2) << 2;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int t = t0 + j;
+                            if (t < T) {
+                                // a plain load: in the dynamic mode other CTAs wrote the factors during this launch
+                                const float sct = per_row ? __fmul_rn(p.row_scale[t], ws) : sc;
+                                float f = __fmul_rn(__int2float_rn(acc[u][j]), sct);
+                                if (has_bias) f = __fadd_rn(f, bv);
+                                y_stage[t * rows + r_local] = narrow1<BF>(f);
+                                if (acc_n != nullptr) acc_n[(size_t)t * N] = acc[u][j];
+                            }
+                        }
+                    }
+                }
+            }
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        {
+            const int vec_per_token = rows >> 3;                          // rows >= 16: whole groups of 8 channels
+            const int vecs = T * vec_per_token;
+            const int n_first = n0 + rank * rows;
+            uint16_t* y = reinterpret_cast<uint16_t*>(p.y);
+            for (int v = et; v < vecs; v += 128) {
+                const int t = v / vec_per_token, c8 = v - t * vec_per_token;
+                const int nn = n_first + 8 * c8;
+                if (nn < p.N)                                             // N % 8 == 0: a group is inside or outside
+                    *reinterpret_cast<uint4*>(y + (size_t)t * N + nn) =
+                        *reinterpret_cast<const uint4*>(y_stage + t * rows + 8 * c8);
             }
         }
     }
