@@ -162,6 +162,17 @@ __device__ __forceinline__ void local_activation_tiles(const DecodeParams& dp, c
     }
 }
 
+// fl32(a) for a 32-bit integer, round to nearest even (what cvt.rn.f32.s32 returns), on the integer and FMA pipes:
+// a = hi * 2^16 + lo with hi in [-2^15, 2^15) and lo in [0, 2^16); each half becomes a float exactly by adding it to
+// the mantissa of a constant and subtracting the constant, and one fused multiply-add rounds hi * 65536 + lo, which
+// is a itself, once.  The conversion pipe takes about 30 cycles per warp instruction here (measured: 135 cycles per
+// output with two conversions each), and in this kernel's last phase a warp has nothing else to overlap them with.
+__device__ __forceinline__ float int_to_float_exact(int a) {
+    const float hi = __fsub_rn(__int_as_float(0x4B400000 + (a >> 16)), 12582912.0f);                     // 1.5 * 2^23 + hi
+    const float lo = __fsub_rn(__uint_as_float(0x4B000000u | ((unsigned)a & 0xFFFFu)), 8388608.0f);      // 2^23 + lo
+    return __fmaf_rn(hi, 65536.0f, lo);
+}
+
 template <bool BF>
 __global__ void __launch_bounds__(D_THREADS, 1)
 w8a8_decode_kernel(const __grid_constant__ DecodeMaps maps, const __grid_constant__ DecodeParams dp) {
@@ -525,18 +536,23 @@ w8a8_decode_kernel(const __grid_constant__ DecodeMaps maps, const __grid_constan
                     const int it = it0 + 128 * u;
                     if (it < items) {
                         const int t0 = (it >> rows_log2) << 2;
+                        float f[4];
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             const int t = t0 + j;
-                            if (t < T) {
-                                // a plain load: in the dynamic mode other CTAs wrote the factors during this launch
-                                const float sct = per_row ? __fmul_rn(p.row_scale[t], ws) : sc;
-                                float f = __fmul_rn(__int2float_rn(acc[u][j]), sct);
-                                if (has_bias) f = __fadd_rn(f, bv);
-                                y_stage[t * rows + r_local] = narrow1<BF>(f);
-                                if (acc_n != nullptr) acc_n[(size_t)t * N] = acc[u][j];
-                            }
+                            // a plain load: in the dynamic mode other CTAs wrote the factors during this launch
+                            const float sct = (per_row && t < T) ? __fmul_rn(p.row_scale[t], ws) : sc;
+                            f[j] = __fmul_rn(int_to_float_exact(acc[u][j]), sct);
+                            if (has_bias) f[j] = __fadd_rn(f[j], bv);
+                            if (acc_n != nullptr && t < T) acc_n[(size_t)t * N] = acc[u][j];
                         }
+                        // two values per narrowing instruction; rows t >= T of the staging tile are never copied out
+                        const uint32_t lo = narrow2<BF>(f[0], f[1]), hi = narrow2<BF>(f[2], f[3]);
+                        uint16_t* dst = y_stage + t0 * rows + r_local;
+                        dst[0] = (uint16_t)(lo & 0xFFFFu);
+                        dst[rows] = (uint16_t)(lo >> 16);
+                        dst[2 * rows] = (uint16_t)(hi & 0xFFFFu);
+                        dst[3 * rows] = (uint16_t)(hi >> 16);
                     }
                 }
             }
