@@ -344,7 +344,7 @@ def linears_by_calls(P, stack, tokens: int, seconds: float, modes=("each", "depe
     """The seven static linears of a layer at `tokens` rows, back to back, for each way of submitting them; the
     layers' weights take turns so that no repetition finds its weights in L2.  graph: the calls of up to eight
     layers are captured once into a CUDA graph and the graph is replayed, which takes the host's per-call cost
-    (a few microseconds, more than a decode-sized kernel runs) out of the measurement; times are per layer."""
+    (about 5 us, of the order of a decode-sized kernel) out of the measurement; times are per layer."""
     ops = linear_ops(tokens)
     out = {}
     for name in modes:
