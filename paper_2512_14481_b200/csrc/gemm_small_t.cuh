@@ -499,77 +499,107 @@ w8a8_decode_kernel(const __grid_constant__ DecodeMaps maps, const __grid_constan
         const float ws = pre_ws;
         const float sc = __fmul_rn(sx, ws);
         const float bv = pre_bias;
-        // Four items at a time: first all their slot reads (explicit shared-memory loads: through generic pointers the
-        // compiler would have to keep every read behind the global stores before it), then their outputs, so that
-        // the latencies of the conversions and of the address arithmetic overlap instead of adding up (a thread has
-        // up to 32 items and a warp has the SM sub-partition to itself).
-        const int rows_log2 = 31 - __clz(rows);                 // rows is a power of two
-        const uint32_t slots_s = ptx::smem_u32(ring) + (uint32_t)dp.slots_offset;
-        // The outputs of the CTA (T tokens x rows channels) are gathered in shared memory, [token][channel], and then
-        // written with 128-bit stores: 2-byte stores, one channel per lane and one token per instruction, were the
-        // longest phase of a 128-row launch (13 us of 33 for 128 channels).  The pipeline stages are free by now:
-        // the accumulators this warp read were complete, so every load had landed and every MMA had read it.
-        uint16_t* y_stage = reinterpret_cast<uint16_t*>(ring);
-        int32_t* acc_n = p.acc_out != nullptr ? p.acc_out + n : nullptr;
-        const int T = p.T;
-        const size_t N = (size_t)p.N;
-        for (int it0 = et; it0 < items; it0 += 4 * 128) {
-            int32_t acc[4][4];
+        if (dp.tp <= 80) {
+            // Up to 80 rows the outputs are written directly, 2 bytes per lane: the gathered form below costs a
+            // barrier and a second pass and only pays from 96 rows up (measured, same run: 16 rows 77 against 85 us
+            // for a layer's four dependent calls, 48 rows 85 against 91, 96 rows and up 2 to 10 % the other way).
+            const int32_t* slots = reinterpret_cast<const int32_t*>(ring + dp.slots_offset);
+            for (int it = et; it < items; it += 128) {
+                const int t0 = (it / rows) << 2;
+                int32_t acc[4] = {0, 0, 0, 0};
+                for (int r = 0; r < dp.split; ++r) {
+                    const int4 v = *reinterpret_cast<const int4*>(slots + (size_t)(r * rows + r_local) * pstride + t0);
+                    acc[0] += v.x; acc[1] += v.y; acc[2] += v.z; acc[3] += v.w;
+                }
+                if (n < p.N) {
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int it = it0 + 128 * u;
-                acc[u][0] = acc[u][1] = acc[u][2] = acc[u][3] = 0;
-                if (it < items) {
-                    const int t0 = (it >> rows_log2) << 2;
-                    for (int r = 0; r < dp.split; ++r) {
-                        int4 v;
-                        asm volatile("ld.shared.v4.s32 {%0, %1, %2, %3}, [%4];"
-                                     : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                                     : "r"(slots_s + (uint32_t)(((r << rows_log2) + r_local) * pstride + t0) * 4u));
-                        acc[u][0] += v.x; acc[u][1] += v.y; acc[u][2] += v.z; acc[u][3] += v.w;
+                    for (int j = 0; j < 4; ++j) {
+                        const int t = t0 + j;
+                        if (t < p.T) {
+                            // a plain load: in the dynamic mode other CTAs wrote the factors during this launch
+                            const float sct = per_row ? __fmul_rn(p.row_scale[t], ws) : sc;
+                            float f = __fmul_rn(__int2float_rn(acc[j]), sct);
+                            if (has_bias) f = __fadd_rn(f, bv);
+                            reinterpret_cast<uint16_t*>(p.y)[(size_t)t * p.N + n] = narrow1<BF>(f);
+                            if (p.acc_out != nullptr) p.acc_out[(size_t)t * p.N + n] = acc[j];
+                        }
                     }
                 }
             }
-            if (n < p.N) {
+        } else {
+            // Four items at a time: first all their slot reads (explicit shared-memory loads: through generic pointers the
+            // compiler would have to keep every read behind the global stores before it), then their outputs, so that
+            // the latencies of the conversions and of the address arithmetic overlap instead of adding up (a thread has
+            // up to 32 items and a warp has the SM sub-partition to itself).
+            const int rows_log2 = 31 - __clz(rows);                 // rows is a power of two
+            const uint32_t slots_s = ptx::smem_u32(ring) + (uint32_t)dp.slots_offset;
+            // The outputs of the CTA (T tokens x rows channels) are gathered in shared memory, [token][channel], and then
+            // written with 128-bit stores: 2-byte stores, one channel per lane and one token per instruction, were the
+            // longest phase of a 128-row launch (13 us of 33 for 128 channels).  The pipeline stages are free by now:
+            // the accumulators this warp read were complete, so every load had landed and every MMA had read it.
+            uint16_t* y_stage = reinterpret_cast<uint16_t*>(ring);
+            int32_t* acc_n = p.acc_out != nullptr ? p.acc_out + n : nullptr;
+            const int T = p.T;
+            const size_t N = (size_t)p.N;
+            for (int it0 = et; it0 < items; it0 += 4 * 128) {
+                int32_t acc[4][4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const int it = it0 + 128 * u;
+                    acc[u][0] = acc[u][1] = acc[u][2] = acc[u][3] = 0;
                     if (it < items) {
                         const int t0 = (it >> rows_log2) << 2;
-                        float f[4];
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const int t = t0 + j;
-                            // a plain load: in the dynamic mode other CTAs wrote the factors during this launch
-                            const float sct = (per_row && t < T) ? __fmul_rn(p.row_scale[t], ws) : sc;
-                            f[j] = __fmul_rn(int_to_float_exact(acc[u][j]), sct);
-                            if (has_bias) f[j] = __fadd_rn(f[j], bv);
-                            if (acc_n != nullptr && t < T) acc_n[(size_t)t * N] = acc[u][j];
+                        for (int r = 0; r < dp.split; ++r) {
+                            int4 v;
+                            asm volatile("ld.shared.v4.s32 {%0, %1, %2, %3}, [%4];"
+                                         : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                                         : "r"(slots_s + (uint32_t)(((r << rows_log2) + r_local) * pstride + t0) * 4u));
+                            acc[u][0] += v.x; acc[u][1] += v.y; acc[u][2] += v.z; acc[u][3] += v.w;
                         }
-                        // two values per narrowing instruction; rows t >= T of the staging tile are never copied out
-                        const uint32_t lo = narrow2<BF>(f[0], f[1]), hi = narrow2<BF>(f[2], f[3]);
-                        uint16_t* dst = y_stage + t0 * rows + r_local;
-                        dst[0] = (uint16_t)(lo & 0xFFFFu);
-                        dst[rows] = (uint16_t)(lo >> 16);
-                        dst[2 * rows] = (uint16_t)(hi & 0xFFFFu);
-                        dst[3 * rows] = (uint16_t)(hi >> 16);
+                    }
+                }
+                if (n < p.N) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int it = it0 + 128 * u;
+                        if (it < items) {
+                            const int t0 = (it >> rows_log2) << 2;
+                            float f[4];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const int t = t0 + j;
+                                // a plain load: in the dynamic mode other CTAs wrote the factors during this launch
+                                const float sct = (per_row && t < T) ? __fmul_rn(p.row_scale[t], ws) : sc;
+                                f[j] = __fmul_rn(int_to_float_exact(acc[u][j]), sct);
+                                if (has_bias) f[j] = __fadd_rn(f[j], bv);
+                                if (acc_n != nullptr && t < T) acc_n[(size_t)t * N] = acc[u][j];
+                            }
+                            // two values per narrowing instruction; rows t >= T of the staging tile are never copied out
+                            const uint32_t lo = narrow2<BF>(f[0], f[1]), hi = narrow2<BF>(f[2], f[3]);
+                            uint16_t* dst = y_stage + t0 * rows + r_local;
+                            dst[0] = (uint16_t)(lo & 0xFFFFu);
+                            dst[rows] = (uint16_t)(lo >> 16);
+                            dst[2 * rows] = (uint16_t)(hi & 0xFFFFu);
+                            dst[3 * rows] = (uint16_t)(hi >> 16);
+                        }
                     }
                 }
             }
-        }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        {
-            const int vec_per_token = rows >> 3;                          // rows >= 16: whole groups of 8 channels
-            const int vecs = T * vec_per_token;
-            const int n_first = n0 + rank * rows;
-            uint16_t* y = reinterpret_cast<uint16_t*>(p.y);
-            for (int v = et; v < vecs; v += 128) {
-                const int t = v / vec_per_token, c8 = v - t * vec_per_token;
-                const int nn = n_first + 8 * c8;
-                if (nn < p.N)                                             // N % 8 == 0: a group is inside or outside
-                    *reinterpret_cast<uint4*>(y + (size_t)t * N + nn) =
-                        *reinterpret_cast<const uint4*>(y_stage + t * rows + 8 * c8);
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            {
+                const int vec_per_token = rows >> 3;                          // rows >= 16: whole groups of 8 channels
+                const int vecs = T * vec_per_token;
+                const int n_first = n0 + rank * rows;
+                uint16_t* y = reinterpret_cast<uint16_t*>(p.y);
+                for (int v = et; v < vecs; v += 128) {
+                    const int t = v / vec_per_token, c8 = v - t * vec_per_token;
+                    const int nn = n_first + 8 * c8;
+                    if (nn < p.N)                                             // N % 8 == 0: a group is inside or outside
+                        *reinterpret_cast<uint4*>(y + (size_t)t * N + nn) =
+                            *reinterpret_cast<const uint4*>(y_stage + t * rows + 8 * c8);
+                }
             }
+    
         }
     }
 
