@@ -76,11 +76,17 @@ def workload_name(layers: int, tokens: int) -> str:
 
 def config_of(args) -> dict:
     """The `config` object, the same for both arms."""
-    return {"workload": workload_name(args.layers, args.tokens), "layers": args.layers, "tokens": args.tokens,
-            "bits": BITS, "quantizers": 7 * args.layers,
+    T, L = args.tokens, args.layers
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    return {"workload": workload_name(L, T), "layers": L, "tokens": T,
+            "bits": BITS, "quantizers": 7 * L,
             "phases": "A: fused fake-quant fwd+bwd + scale-gradient reduction, one launch per layer; "
                       "B: static W8A8 linears of every layer",
-            "linear_calls": args.linear_calls}
+            "linear_calls": args.linear_calls,
+            "l2": f"inputs larger than L2: {quantizer_bytes(T) / 1e6:.0f} MB streamed per layer in phase A, "
+                  f"{(weight_bytes() + 2 * quantizer_elements(T)) / 1e6:.0f} MB of weights+activations per "
+                  f"layer in phase B, {L} layers with their own weights",
+            "parallelism": "replicas" if world > 1 else "single"}
 
 
 def measured_peaks():
@@ -578,12 +584,8 @@ def run_ours(args):
         "warmup": warmup, "ms_per_step": round(ms_total / K, 5), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 storage, fp32 quantizer arithmetic, int8 x int8 -> int32 GEMM", "data": "synthetic",
-        "config": dict(config_of(args),
-                       l2=f"inputs larger than L2: {quantizer_bytes(T) / 1e6:.0f} MB streamed per layer in phase A, "
-                          f"{(weight_bytes() + 2 * quantizer_elements(T)) / 1e6:.0f} MB of weights+activations per "
-                          f"layer in phase B, {L} layers with their own weights",
-                       launch_mode="single stream, plain launches (sasq_set_gang_launch(0))",
-                       parallelism="replicas" if world > 1 else "single"),
+        "config": config_of(args),
+        "launch_mode": "single stream, plain launches (sasq_set_gang_launch(0))",
         "ms_phase_a": round(ms_a / K, 5), "ms_phase_b": round(ms_b / K, 5),
         "phase_stats": {"steps_seen": len(extra_a),
                         "a_ms_median": round(statistics.median(extra_a), 5), "a_ms_min": round(min(extra_a), 5),
