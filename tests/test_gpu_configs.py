@@ -185,3 +185,53 @@ def test_config5_full_stack_scale_only_step_then_static_prefill():
                     assert np.array_equal(host_bits(ys[i]), y_o) and np.array_equal(host_bits(dxs[i]), dx_o)
     assert ds_checked == 21
     assert bool((grads != 3.0).all())          # every one of the 224 slots was written
+
+
+def test_config5_one_layer_in_the_launch_configuration_the_benchmark_times():
+    """One layer of config 5 (T = 16 384) submitted exactly as the benchmark's step submits it: the fused fake-quant
+    forward + backward of the seven inputs as ONE prepared multi-tensor call, then the seven static linears in the
+    groups a decoder layer's data flow allows (q/k/v | o | gate/up | down) as prepared multi-linear calls, plain
+    (not co-operative) launches, raw stream handle.  Every scale gradient against the oracle's double sum, two
+    tensors element by element, sampled rows of every linear bit for bit."""
+    tag, T, bits = oracle.BF16, 8 * 2048, 8
+    shapes = [(K, N) for _, K, N in W.LLAMA2_7B_LINEARS]
+    xs = [W.activations(T, K, torch.bfloat16, W.seed_of(5, 500 + i), device="cuda") for i, (K, _) in enumerate(shapes)]
+    gs = [W.upstream_grad(T, K, torch.bfloat16, W.seed_of(5, 500 + i), device="cuda") for i, (K, _) in enumerate(shapes)]
+    ys, dxs = [torch.empty_like(t) for t in xs], [torch.empty_like(t) for t in xs]
+    outs = [torch.empty((T, N), dtype=torch.bfloat16, device="cuda") for _, N in shapes]
+    weights = [device_weights(N, K, W.seed_of(5, 600 + i)) for i, (K, N) in enumerate(shapes)]
+    scales = torch.empty(7, dtype=torch.float32, device="cuda")
+    grads = torch.zeros(7, dtype=torch.float32, device="cuda")
+    cal_ws = torch.empty(P.sasq_absmax_scale_workspace(0), dtype=torch.uint8, device="cuda")
+    for i in range(7):
+        P.sasq_absmax_scale(xs[i][:W.CALIBRATION_TOKENS], scales[i:i + 1], cal_ws, bits)
+    q_ws = torch.empty(P.sasq_fakequant_multi_workspace(7), dtype=torch.uint8, device="cuda")
+    l_ws = torch.empty(P.sasq_static_w8a8_linear_multi_workspace([(T, N, K) for K, N in shapes]), dtype=torch.uint8,
+                       device="cuda")
+    quant = P.QuantTensors([(xs[i], gs[i], ys[i], dxs[i], i) for i in range(7)])
+    calls = [P.LinearProblems([(xs[i], weights[i][0], weights[i][1], scales[i:i + 1], outs[i]) for i in call])
+             for call in ([0, 1, 2], [3], [4, 5], [6])]
+    handle = torch.cuda.current_stream().cuda_stream
+    previous = P.sasq_set_gang_launch(False)
+    try:
+        for _ in range(2):                                  # twice: the second pass finds the counters as the first left them
+            P.sasq_fakequant_fwd_bwd_multi(quant, scales, grads, q_ws, bits, stream=handle)
+            for problems in calls:
+                P.sasq_static_w8a8_linear_multi(problems, l_ws, bits=bits, stream=handle)
+        assert P.sasq_device_status() == 0
+    finally:
+        P.sasq_set_gang_launch(previous)
+    s_host = scales.cpu().numpy()
+    for i, (K, N) in enumerate(shapes):
+        s = float(s_host[i])
+        xb, gb = host_bits(xs[i]), host_bits(gs[i])
+        dx_o, ds_o = oracle.fakequant_bwd(xb, gb, tag, s, bits)
+        assert abs(grads[i].item() - ds_o) <= DS_RTOL * abs(ds_o), i
+        if i in (1, 6):
+            y_o, _ = oracle.fakequant_fwd(xb, tag, s, bits, want_codes=False)
+            assert np.array_equal(host_bits(ys[i]), y_o) and np.array_equal(host_bits(dxs[i]), dx_o), i
+        rows = sample_rows(T, 700 + i, n_random=3)
+        idx = torch.tensor(rows, device="cuda")
+        y_lin, _, _ = oracle.w8a8_linear(oracle.bits_of(xs[i][idx].cpu())[0], tag, weights[i][0].cpu().numpy(),
+                                         weights[i][1].cpu().numpy(), s, bits)
+        assert np.array_equal(host_bits(outs[i][idx]), y_lin), i
