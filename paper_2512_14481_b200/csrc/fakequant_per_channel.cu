@@ -112,9 +112,15 @@ __global__ void __launch_bounds__(kPcThreads, kPcBlocksPerSM) fakequant_pc_kerne
                 if constexpr (BWD) gv[u] = pc_load(d.g + r * vec_per_row + cv);
             }
         }
+        // the products of the rows in flight are first added in fp32, in a fixed tree, and reach the double sums
+        // once per trip: a float -> double conversion and a double add per ELEMENT kept the conversion pipe busier
+        // than the memory system (the per-tensor kernel likewise adds a vector's 8 products in fp32 first)
+        float prod[UNROLL][8];
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
             const long long r = r0 + (long long)u * n_rg;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) prod[u][j] = 0.0f;
             if (r < T) {
                 const uint32_t xw[4] = {xv[u].x, xv[u].y, xv[u].z, xv[u].w};
                 uint32_t gw[4] = {0u, 0u, 0u, 0u};
@@ -133,12 +139,25 @@ __global__ void __launch_bounds__(kPcThreads, kPcBlocksPerSM) fakequant_pc_kerne
                         const float2 gf = widen2<BF>(gw[q]);
                         const bool in0 = (c0 == r_0), in1 = (c1 == r_1);      // false for NaN as well
                         dxo[q] = (in0 ? (gw[q] & 0x0000FFFFu) : 0u) | (in1 ? (gw[q] & 0xFFFF0000u) : 0u);
-                        acc[2 * q] += (double)__fmul_rn(gf.x, in0 ? __fsub_rn(r_0, t0) : c0);
-                        acc[2 * q + 1] += (double)__fmul_rn(gf.y, in1 ? __fsub_rn(r_1, t1) : c1);
+                        prod[u][2 * q] = __fmul_rn(gf.x, in0 ? __fsub_rn(r_0, t0) : c0);
+                        prod[u][2 * q + 1] = __fmul_rn(gf.y, in1 ? __fsub_rn(r_1, t1) : c1);
                     }
                 }
                 if constexpr (FWD) pc_store(d.y + r * vec_per_row + cv, make_uint4(yo[0], yo[1], yo[2], yo[3]));
                 if constexpr (BWD) pc_store(d.dx + r * vec_per_row + cv, make_uint4(dxo[0], dxo[1], dxo[2], dxo[3]));
+            }
+        }
+        if constexpr (BWD) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                float sum = 0.0f;
+                if constexpr (UNROLL == 4) {
+                    sum = __fadd_rn(__fadd_rn(prod[0][j], prod[1][j]), __fadd_rn(prod[2][j], prod[3][j]));
+                } else {
+#pragma unroll
+                    for (int u = 0; u < UNROLL; ++u) sum = __fadd_rn(sum, prod[u][j]);
+                }
+                acc[j] += (double)sum;
             }
         }
     }
